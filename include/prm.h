@@ -1,0 +1,147 @@
+/*
+ * prm.h - C ABI of the Periodic Row-wise Muon optimizer step for NVIDIA B200.
+ *
+ * The library performs, for a list of 2-D weight matrices, the matrix branch
+ * of the paper's Algorithm 1 ("Periodic Row-wise Muon"): momentum update,
+ * orientation, then either the NS5 spectral refresh (Eq. periodic-direction,
+ * rho_t = 1; recurrence of Appendix Eq. app-ns-recurrence) or the row-wise
+ * normalised direction gamma * RowNorm_eps (Eq. rownorm, rho_t = 0), and the
+ * decoupled-weight-decay parameter update of Eq. periodic-direction.
+ *
+ * Conventions
+ *   - Matrices are stored row-major, contiguous, rows x cols; "wide" means
+ *     rows <= cols, "tall" means rows > cols.  The orientation map of
+ *     Section 3.1 transposes tall matrices, so RowNorm normalises stored
+ *     rows of wide matrices and stored COLUMNS of tall ones.
+ *   - All matrix pointers are DEVICE pointers, 16-byte aligned.  The arrays
+ *     of pointers handed to prm_step are HOST arrays of length n_mats.
+ *   - The caller owns parameters, gradients, momentum, the workspace and the
+ *     stream.  prm_step enqueues work on the stream and returns; it never
+ *     synchronises and never allocates device memory.
+ *   - Every function returns PRM_OK (0) or a negative error code; nothing
+ *     aborts the process.  prm_last_error() gives a text for the last error
+ *     on that handle.
+ *   - There is no CPU fallback: without a CUDA device the compute entry
+ *     points return PRM_ERR_CUDA.
+ */
+#ifndef PRM_H_
+#define PRM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define PRM_API __attribute__((visibility("default")))
+#else
+#define PRM_API
+#endif
+
+#define PRM_OK                  0
+#define PRM_ERR_ARG            -1   /* null pointer, K < 1, bad option key or value */
+#define PRM_ERR_SHAPE          -2   /* non-positive or unsupported dimension */
+#define PRM_ERR_ALIGN          -3   /* device pointer not 16-byte aligned */
+#define PRM_ERR_WORKSPACE      -4   /* workspace missing or too small */
+#define PRM_ERR_CUDA           -5   /* a CUDA runtime/driver call failed */
+#define PRM_ERR_DEVICE_TIMEOUT -6   /* a bounded device-side wait expired */
+#define PRM_ERR_STATE          -7   /* call not allowed in this state */
+
+/* Option keys for prm_set_option. */
+#define PRM_OPT_GAMMA        1  /* RowNorm multiplier gamma (Section 3.2), default 0.15 */
+#define PRM_OPT_EPS_ROW      2  /* epsilon of Eq. rownorm, default 1e-8 */
+#define PRM_OPT_EPS_NS       3  /* epsilon added to ||X||_F before NS5, default 1e-7 */
+#define PRM_OPT_SCALE_MODE   4  /* s(W): 0 -> 1; 1 (default) -> sqrt(max(1, rows/cols));
+                                   2 -> 0.2*sqrt(max(rows, cols)) */
+#define PRM_OPT_IO_DTYPE     5  /* 0 (default): bf16 params and grads; 1: fp32 params and
+                                   grads.  Momentum is fp32 in both.  Before set_workspace. */
+#define PRM_OPT_CHECK_MODE   6  /* 0 (default): NS5 on tensor cores, bf16 operands, fp32
+                                   accumulate; 1: NS5 in fp32 on CUDA cores (slow, for
+                                   verification).  Before set_workspace. */
+#define PRM_OPT_LR           7  /* eta_t; may be changed between any two steps */
+#define PRM_OPT_WD           8  /* lambda; may be changed between any two steps */
+#define PRM_OPT_NS_WORKSPACE_BYTES 9 /* soft cap on the NS5 part of the workspace, default
+                                   8 GiB; matrices of one shape group are refreshed in
+                                   sub-batches that fit.  Before set_workspace. */
+
+typedef struct prm_ctx prm_ctx;
+
+/*
+ * Create a handle for n_mats matrices (Algorithm 1's Muon set W_M).
+ *   shapes   host array of 2*n_mats int64: (rows, cols) of matrix i at [2i], [2i+1]
+ *   K        refresh period, K >= 1; step t refreshes iff t mod K == 0 (Section 3.2)
+ *   beta     momentum coefficient of M_t = beta*M_{t-1} + (1-beta)*G_t
+ *   nesterov 0: direction from M_t; 1: from beta*M_t + (1-beta)*G_t
+ *   lr, wd   eta_t and lambda of Eq. periodic-direction
+ * Uses the CUDA device current at the time of the call.  Allocates only host
+ * memory.  On failure *out is NULL.
+ */
+PRM_API int prm_create(prm_ctx** out, const int64_t* shapes, int n_mats,
+               int K, float beta, int nesterov, float lr, float wd);
+
+/* Set an option (keys above).  Returns PRM_ERR_STATE for options that must be
+ * set before prm_set_workspace once a workspace is attached. */
+PRM_API int prm_set_option(prm_ctx* ctx, int key, double value);
+
+/* Bytes of device workspace needed with the current options (pointer tables,
+ * column-norm scratch of tall row-steps, NS5 operands).  0 on a NULL handle. */
+PRM_API size_t prm_workspace_bytes(const prm_ctx* ctx);
+
+/* Attach caller-allocated device workspace (256-byte aligned, at least
+ * prm_workspace_bytes).  The library keeps the pointer until prm_destroy or
+ * the next prm_set_workspace; the caller frees it afterwards. */
+PRM_API int prm_set_workspace(prm_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/*
+ * One optimizer step for all matrices (Algorithm 1 lines 2-9 for step t =
+ * step_idx, zero-based): updates momentum[i] and params[i] in place, reads
+ * grads[i].  params/grads: bf16 or fp32 per PRM_OPT_IO_DTYPE; momentum: fp32.
+ * The branch depends only on step_idx mod K; steps need not be consecutive.
+ * cuda_stream is a cudaStream_t (NULL = default stream).  Calls on one handle
+ * must be ordered on one stream, or separated by synchronisation.
+ */
+PRM_API int prm_step(prm_ctx* ctx, void* const* params, const void* const* grads,
+             float* const* momentum, int64_t step_idx, void* cuda_stream);
+
+/*
+ * Same step, but first copies this step's gradients from HOST memory:
+ * grads_host[i] (rows*cols elements of the I/O dtype, ideally pinned) is
+ * copied to grads_dev[i] with one asynchronous copy per matrix on the stream,
+ * then the step runs as in prm_step.
+ */
+PRM_API int prm_step_h2d(prm_ctx* ctx, void* const* params, void* const* grads_dev,
+                 const void* const* grads_host, float* const* momentum,
+                 int64_t step_idx, void* cuda_stream);
+
+/*
+ * The schedule and the shape grouping, without touching the device.
+ *   is_refresh      1 iff step_idx mod K == 0
+ *   n_groups        number of distinct (rows, cols) pairs
+ *   group_of_mat    [n_mats] group id, ids numbered by first appearance
+ *   order_in_group  [n_mats] position inside the group, caller order kept
+ * Any output pointer may be NULL.
+ */
+PRM_API int prm_plan(const prm_ctx* ctx, int64_t step_idx, int* is_refresh,
+             int* n_groups, int* group_of_mat, int* order_in_group);
+
+/* Reads the device status word (synchronises the device first): PRM_OK, or
+ * PRM_ERR_DEVICE_TIMEOUT if a kernel gave up on a bounded wait since the last
+ * call; the word is cleared. */
+PRM_API int prm_status(prm_ctx* ctx);
+
+/* Text of the last error on this handle ("" if none).  Valid until the next
+ * call on the handle.  With ctx == NULL: the last prm_create error. */
+PRM_API const char* prm_last_error(const prm_ctx* ctx);
+
+/* Number of kernels the library has launched through this handle so far. */
+PRM_API int64_t prm_launch_count(const prm_ctx* ctx);
+
+/* Frees host resources.  Device memory belongs to the caller. */
+PRM_API int prm_destroy(prm_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PRM_H_ */

@@ -1,0 +1,238 @@
+"""ctypes binding of the prm C ABI (include/prm.h).
+
+Argument marshalling only: every arithmetic step runs in the CUDA library.
+The functions carry the C names; `PeriodicRowwiseMuon` bundles a handle with
+a torch-allocated workspace.  Loading fails loudly when libprm.so is missing;
+there is no fallback path.
+"""
+
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_double, c_float, c_int, c_int64, c_size_t, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libprm.so")
+
+PRM_OK = 0
+PRM_ERR_ARG = -1
+PRM_ERR_SHAPE = -2
+PRM_ERR_ALIGN = -3
+PRM_ERR_WORKSPACE = -4
+PRM_ERR_CUDA = -5
+PRM_ERR_DEVICE_TIMEOUT = -6
+PRM_ERR_STATE = -7
+
+PRM_OPT_GAMMA = 1
+PRM_OPT_EPS_ROW = 2
+PRM_OPT_EPS_NS = 3
+PRM_OPT_SCALE_MODE = 4
+PRM_OPT_IO_DTYPE = 5
+PRM_OPT_CHECK_MODE = 6
+PRM_OPT_LR = 7
+PRM_OPT_WD = 8
+PRM_OPT_NS_WORKSPACE_BYTES = 9
+
+EXPORTS = (
+    "prm_create", "prm_set_option", "prm_workspace_bytes", "prm_set_workspace", "prm_step",
+    "prm_step_h2d", "prm_plan", "prm_status", "prm_last_error", "prm_launch_count", "prm_destroy",
+)
+
+_lib_handle = None
+
+
+class PrmError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"prm error {code}: {msg}")
+        self.code = code
+
+
+def lib():
+    """The loaded CUDA library.  Raises if it has not been built."""
+    global _lib_handle
+    if _lib_handle is not None:
+        return _lib_handle
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2608_20818_b200.build` "
+            "(nvcc, sm_100a). There is no CPU fallback.")
+    L = ctypes.CDLL(LIB_PATH)
+    L.prm_create.argtypes = [POINTER(c_void_p), POINTER(c_int64), c_int, c_int, c_float, c_int, c_float, c_float]
+    L.prm_create.restype = c_int
+    L.prm_set_option.argtypes = [c_void_p, c_int, c_double]
+    L.prm_set_option.restype = c_int
+    L.prm_workspace_bytes.argtypes = [c_void_p]
+    L.prm_workspace_bytes.restype = c_size_t
+    L.prm_set_workspace.argtypes = [c_void_p, c_void_p, c_size_t]
+    L.prm_set_workspace.restype = c_int
+    L.prm_step.argtypes = [c_void_p, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p), c_int64, c_void_p]
+    L.prm_step.restype = c_int
+    L.prm_step_h2d.argtypes = [c_void_p, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p),
+                               POINTER(c_void_p), c_int64, c_void_p]
+    L.prm_step_h2d.restype = c_int
+    L.prm_plan.argtypes = [c_void_p, c_int64, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]
+    L.prm_plan.restype = c_int
+    L.prm_status.argtypes = [c_void_p]
+    L.prm_status.restype = c_int
+    L.prm_last_error.argtypes = [c_void_p]
+    L.prm_last_error.restype = c_char_p
+    L.prm_launch_count.argtypes = [c_void_p]
+    L.prm_launch_count.restype = c_int64
+    L.prm_destroy.argtypes = [c_void_p]
+    L.prm_destroy.restype = c_int
+    _lib_handle = L
+    return L
+
+
+def _check(code, handle=None):
+    if code != PRM_OK:
+        msg = lib().prm_last_error(handle)
+        raise PrmError(code, msg.decode() if msg else "")
+
+
+def prm_create(shapes, K, beta, nesterov, lr, wd):
+    flat = []
+    for (m, n) in shapes:
+        flat += [int(m), int(n)]
+    arr = (c_int64 * max(1, len(flat)))(*flat)
+    h = c_void_p()
+    _check(lib().prm_create(byref(h), arr, len(shapes), int(K), float(beta), int(bool(nesterov)), float(lr), float(wd)))
+    return h
+
+
+def prm_set_option(h, key, value):
+    _check(lib().prm_set_option(h, int(key), float(value)), h)
+
+
+def prm_workspace_bytes(h):
+    return int(lib().prm_workspace_bytes(h))
+
+
+def prm_set_workspace(h, dev_ptr, nbytes):
+    _check(lib().prm_set_workspace(h, c_void_p(dev_ptr), nbytes), h)
+
+
+def _ptr_array(tensors):
+    return (c_void_p * len(tensors))(*[t.data_ptr() for t in tensors])
+
+
+def prm_step(h, params, grads, momentum, step_idx, stream=0):
+    """params/grads/momentum: ctypes arrays of device pointers (see ptr_arrays)."""
+    _check(lib().prm_step(h, params, grads, momentum, int(step_idx), c_void_p(stream)), h)
+
+
+def prm_step_h2d(h, params, grads_dev, grads_host, momentum, step_idx, stream=0):
+    _check(lib().prm_step_h2d(h, params, grads_dev, grads_host, momentum, int(step_idx), c_void_p(stream)), h)
+
+
+def prm_plan(h, step_idx, n_mats):
+    is_refresh, n_groups = c_int(), c_int()
+    g = (c_int * n_mats)()
+    o = (c_int * n_mats)()
+    _check(lib().prm_plan(h, int(step_idx), byref(is_refresh), byref(n_groups), g, o), h)
+    return bool(is_refresh.value), n_groups.value, list(g), list(o)
+
+
+def prm_status(h):
+    return int(lib().prm_status(h))
+
+
+def prm_last_error(h):
+    msg = lib().prm_last_error(h)
+    return msg.decode() if msg else ""
+
+
+def prm_launch_count(h):
+    return int(lib().prm_launch_count(h))
+
+
+def prm_destroy(h):
+    _check(lib().prm_destroy(h))
+
+
+class PeriodicRowwiseMuon:
+    """Handle + workspace.  Tensors stay owned by the caller; `step` only
+    marshals their device pointers."""
+
+    def __init__(self, shapes, K, beta=0.95, nesterov=False, lr=5e-3, wd=0.01, *, gamma=0.15,
+                 eps_row=1e-8, eps_ns=1e-7, scale_mode=1, io_dtype="bf16", check_mode=False,
+                 ns_workspace_bytes=None, device="cuda"):
+        self.shapes = [(int(m), int(n)) for (m, n) in shapes]
+        self.device = torch.device(device)
+        self.io_dtype = io_dtype
+        self.h = None
+        with torch.cuda.device(self.device):
+            self.h = prm_create(self.shapes, K, beta, nesterov, lr, wd)
+            prm_set_option(self.h, PRM_OPT_GAMMA, gamma)
+            prm_set_option(self.h, PRM_OPT_EPS_ROW, eps_row)
+            prm_set_option(self.h, PRM_OPT_EPS_NS, eps_ns)
+            prm_set_option(self.h, PRM_OPT_SCALE_MODE, scale_mode)
+            prm_set_option(self.h, PRM_OPT_IO_DTYPE, 1 if io_dtype == "fp32" else 0)
+            prm_set_option(self.h, PRM_OPT_CHECK_MODE, 1 if check_mode else 0)
+            if ns_workspace_bytes is not None:
+                prm_set_option(self.h, PRM_OPT_NS_WORKSPACE_BYTES, ns_workspace_bytes)
+            nbytes = prm_workspace_bytes(self.h)
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            base = (self.workspace.data_ptr() + 255) // 256 * 256
+            prm_set_workspace(self.h, base, nbytes)
+        self._cache_key = None
+        self._arrays = None
+
+    def ptr_arrays(self, params, grads, momentum):
+        key = (tuple(t.data_ptr() for t in params), tuple(t.data_ptr() for t in grads),
+               tuple(t.data_ptr() for t in momentum))
+        if key != self._cache_key:
+            want = torch.float32 if self.io_dtype == "fp32" else torch.bfloat16
+            for i, (p, g, m) in enumerate(zip(params, grads, momentum)):
+                if p.dtype != want or g.dtype != want or m.dtype != torch.float32:
+                    raise TypeError(f"matrix {i}: dtypes must be {want} (params, grads) and float32 (momentum)")
+                if tuple(p.shape) != self.shapes[i] or tuple(g.shape) != self.shapes[i] or tuple(m.shape) != self.shapes[i]:
+                    raise ValueError(f"matrix {i}: shape mismatch")
+                if not (p.is_contiguous() and g.is_contiguous() and m.is_contiguous()):
+                    raise ValueError(f"matrix {i}: tensors must be contiguous")
+            self._arrays = (_ptr_array(params), _ptr_array(grads), _ptr_array(momentum))
+            self._cache_key = key
+        return self._arrays
+
+    def step(self, params, grads, momentum, step_idx, stream=None):
+        """One optimizer step, enqueued on `stream` (default: torch's current stream)."""
+        if len(params) != len(self.shapes):
+            raise ValueError("wrong number of matrices")
+        P, G, M = self.ptr_arrays(params, grads, momentum)
+        s = (stream or torch.cuda.current_stream(self.device)).cuda_stream
+        with torch.cuda.device(self.device):
+            prm_step(self.h, P, G, M, step_idx, s)
+
+    def step_h2d(self, params, grads_dev, grads_host, momentum, step_idx, stream=None):
+        """Step whose gradients are first copied from (pinned) host tensors."""
+        P, G, M = self.ptr_arrays(params, grads_dev, momentum)
+        H = _ptr_array(grads_host)
+        s = (stream or torch.cuda.current_stream(self.device)).cuda_stream
+        with torch.cuda.device(self.device):
+            prm_step_h2d(self.h, P, G, H, M, step_idx, s)
+
+    def set_lr(self, lr):
+        prm_set_option(self.h, PRM_OPT_LR, lr)
+
+    def plan(self, step_idx):
+        return prm_plan(self.h, step_idx, len(self.shapes))
+
+    def status(self):
+        return prm_status(self.h)
+
+    def launch_count(self):
+        return prm_launch_count(self.h)
+
+    def close(self):
+        if self.h is not None:
+            prm_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

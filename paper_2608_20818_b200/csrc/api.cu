@@ -1,0 +1,351 @@
+// C ABI, plan (shape grouping, refresh schedule), workspace layout and the
+// per-step launch sequence.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <algorithm>
+#include <new>
+
+#include "launch.cuh"
+
+using namespace prm;
+
+struct prm_ctx {
+  int n_mats = 0;
+  std::vector<int64_t> shapes;   // 2*n_mats
+  int K = 1;
+  float beta = 0.95f;
+  int nesterov = 0;
+  float lr = 0.f, wd = 0.f;
+  float gamma = 0.15f, eps_row = 1e-8f, eps_ns = 1e-7f;
+  int scale_mode = 1;
+  int io_fp32 = 0;
+  int check_mode = 0;
+  size_t ns_budget = (size_t)8 << 30;
+
+  std::vector<Group> groups;
+  std::vector<int> group_of_mat, order_in_group, slot_of_mat;   // slot = index in pointer tables
+
+  // workspace layout (byte offsets)
+  size_t off_status = 0, off_tables = 0, off_fro = 0, off_alpha = 0, off_ns = 0, total_bytes = 0;
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+  std::vector<void*> host_tables;   // 3*n_mats, grouped order: params | grads | momentum
+  bool tables_uploaded = false;
+
+  TcContext* tc = nullptr;
+  std::string err;
+  int64_t launches = 0;
+};
+
+static std::string g_create_err;
+
+static int fail(prm_ctx* ctx, int code, const std::string& msg) {
+  if (ctx) ctx->err = msg; else g_create_err = msg;
+  return code;
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static float shape_scale(int mode, int64_t rows, int64_t cols) {
+  // s(W) of Eq. finite_ns5: depends on the stored shape only.
+  if (mode == 0) return 1.f;
+  if (mode == 1) return (float)sqrt(std::max(1.0, (double)rows / (double)cols));
+  return (float)(0.2 * sqrt((double)std::max(rows, cols)));
+}
+
+static void compute_layout(prm_ctx* c) {
+  const size_t e = c->check_mode ? 4 : 2;
+  size_t off = 0;
+  c->off_status = off; off += 256;
+  c->off_tables = off; off = align_up(off + (size_t)3 * c->n_mats * sizeof(void*), 256);
+  size_t fro_max = 0, ns_max = 0;
+  int batch_max = 1;
+  for (Group& g : c->groups) {
+    if (g.tall) {
+      const size_t nblk = (size_t)((g.rows + kTallRows - 1) / kTallRows);
+      g.tall_scratch_off = off; off = align_up(off + (size_t)g.count * nblk * g.cols * 4, 256);
+      g.tall_nu_off = off;      off = align_up(off + (size_t)g.count * g.cols * 4, 256);
+    }
+    const size_t per_mat = e * (size_t)(4 * g.rp * g.cp + 2 * g.rp * g.rp);
+    int nb = (int)std::min<size_t>((size_t)g.count, std::max<size_t>(1, c->ns_budget / per_mat));
+    g.ns_batch = nb;
+    ns_max = std::max(ns_max, per_mat * nb);
+    fro_max = std::max(fro_max, (size_t)nb * (size_t)((g.rp / 64) * (g.cp / 64)));
+    batch_max = std::max(batch_max, nb);
+  }
+  c->off_fro = off;   off = align_up(off + fro_max * 4, 256);
+  c->off_alpha = off; off = align_up(off + (size_t)batch_max * 4, 256);
+  c->off_ns = off;    off += ns_max;
+  c->total_bytes = off;
+}
+
+extern "C" int prm_create(prm_ctx** out, const int64_t* shapes, int n_mats, int K, float beta,
+                          int nesterov, float lr, float wd) {
+  if (!out) return fail(nullptr, PRM_ERR_ARG, "prm_create: out is NULL");
+  *out = nullptr;
+  if (!shapes || n_mats < 1) return fail(nullptr, PRM_ERR_ARG, "prm_create: empty shape list");
+  if (K < 1) return fail(nullptr, PRM_ERR_ARG, "prm_create: K must be >= 1");
+  if (!(beta >= 0.f && beta < 1.f)) return fail(nullptr, PRM_ERR_ARG, "prm_create: beta must be in [0,1)");
+  for (int i = 0; i < n_mats; ++i) {
+    const int64_t r = shapes[2 * i], cdim = shapes[2 * i + 1];
+    if (r < 1 || cdim < 1 || r > 0x7fffffffLL || cdim > 0x7fffffffLL)
+      return fail(nullptr, PRM_ERR_SHAPE, "prm_create: dimension out of range");
+    if (round_up(std::min(r, cdim), kPad) > 65536 || round_up(std::max(r, cdim), kPad) > (1 << 22))
+      return fail(nullptr, PRM_ERR_SHAPE, "prm_create: min(rows,cols) > 65536 or max > 4194304 unsupported");
+  }
+  prm_ctx* c = new (std::nothrow) prm_ctx();
+  if (!c) return fail(nullptr, PRM_ERR_ARG, "prm_create: out of host memory");
+  c->n_mats = n_mats;
+  c->shapes.assign(shapes, shapes + 2 * n_mats);
+  c->K = K; c->beta = beta; c->nesterov = nesterov ? 1 : 0; c->lr = lr; c->wd = wd;
+  // Grouping: exact (rows, cols); ids by first appearance; caller order inside.
+  c->group_of_mat.resize(n_mats);
+  c->order_in_group.resize(n_mats);
+  for (int i = 0; i < n_mats; ++i) {
+    const int64_t r = shapes[2 * i], cdim = shapes[2 * i + 1];
+    int gi = -1;
+    for (size_t k = 0; k < c->groups.size(); ++k)
+      if (c->groups[k].rows == r && c->groups[k].cols == cdim) { gi = (int)k; break; }
+    if (gi < 0) {
+      Group g;
+      g.rows = r; g.cols = cdim; g.tall = r > cdim;
+      g.r = std::min(r, cdim); g.c = std::max(r, cdim);
+      g.rp = round_up(g.r, kPad); g.cp = round_up(g.c, kPad);
+      c->groups.push_back(g);
+      gi = (int)c->groups.size() - 1;
+    }
+    c->group_of_mat[i] = gi;
+    c->order_in_group[i] = c->groups[gi].count++;
+  }
+  int first = 0;
+  for (Group& g : c->groups) { g.first = first; first += g.count; }
+  c->slot_of_mat.resize(n_mats);
+  for (int i = 0; i < n_mats; ++i)
+    c->slot_of_mat[i] = c->groups[c->group_of_mat[i]].first + c->order_in_group[i];
+  c->host_tables.assign((size_t)3 * n_mats, nullptr);
+  compute_layout(c);
+  *out = c;
+  return PRM_OK;
+}
+
+extern "C" int prm_set_option(prm_ctx* c, int key, double v) {
+  if (!c) return PRM_ERR_ARG;
+  const bool attached = c->ws != nullptr;
+  switch (key) {
+    case PRM_OPT_GAMMA: if (!(v > 0)) return fail(c, PRM_ERR_ARG, "gamma must be > 0"); c->gamma = (float)v; return PRM_OK;
+    case PRM_OPT_EPS_ROW: if (v < 0) return fail(c, PRM_ERR_ARG, "eps_row must be >= 0"); c->eps_row = (float)v; return PRM_OK;
+    case PRM_OPT_EPS_NS: if (v < 0) return fail(c, PRM_ERR_ARG, "eps_ns must be >= 0"); c->eps_ns = (float)v; return PRM_OK;
+    case PRM_OPT_SCALE_MODE:
+      if (v != 0 && v != 1 && v != 2) return fail(c, PRM_ERR_ARG, "scale mode must be 0, 1 or 2");
+      c->scale_mode = (int)v; return PRM_OK;
+    case PRM_OPT_LR: c->lr = (float)v; return PRM_OK;
+    case PRM_OPT_WD: c->wd = (float)v; return PRM_OK;
+    case PRM_OPT_IO_DTYPE:
+    case PRM_OPT_CHECK_MODE:
+    case PRM_OPT_NS_WORKSPACE_BYTES:
+      if (attached) return fail(c, PRM_ERR_STATE, "option must be set before prm_set_workspace");
+      if (key == PRM_OPT_NS_WORKSPACE_BYTES) {
+        if (v < 0) return fail(c, PRM_ERR_ARG, "workspace cap must be >= 0");
+        c->ns_budget = (size_t)v;
+      } else {
+        if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
+        (key == PRM_OPT_IO_DTYPE ? c->io_fp32 : c->check_mode) = (int)v;
+      }
+      compute_layout(c);
+      return PRM_OK;
+    default: return fail(c, PRM_ERR_ARG, "unknown option key");
+  }
+}
+
+extern "C" size_t prm_workspace_bytes(const prm_ctx* c) { return c ? c->total_bytes : 0; }
+
+extern "C" int prm_set_workspace(prm_ctx* c, void* dev_ptr, size_t bytes) {
+  if (!c) return PRM_ERR_ARG;
+  if (!dev_ptr) return fail(c, PRM_ERR_ARG, "prm_set_workspace: NULL pointer");
+  if (((uintptr_t)dev_ptr & 255) != 0) return fail(c, PRM_ERR_ALIGN, "prm_set_workspace: pointer not 256-byte aligned");
+  if (bytes < c->total_bytes) return fail(c, PRM_ERR_WORKSPACE, "prm_set_workspace: workspace too small");
+  cudaError_t e = cudaMemset(dev_ptr, 0, 256);
+  if (e != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("prm_set_workspace: ") + cudaGetErrorString(e));
+  c->ws = (char*)dev_ptr;
+  c->ws_bytes = bytes;
+  c->tables_uploaded = false;
+  if (!c->check_mode && !c->tc) {
+    std::string err;
+    c->tc = tc_create(&err);
+    if (!c->tc) { c->ws = nullptr; return fail(c, PRM_ERR_CUDA, "prm_set_workspace: " + err); }
+  }
+  return PRM_OK;
+}
+
+extern "C" int prm_plan(const prm_ctx* c, int64_t step_idx, int* is_refresh, int* n_groups,
+                        int* group_of_mat, int* order_in_group) {
+  if (!c || step_idx < 0) return PRM_ERR_ARG;
+  if (is_refresh) *is_refresh = (step_idx % c->K) == 0 ? 1 : 0;
+  if (n_groups) *n_groups = (int)c->groups.size();
+  if (group_of_mat) memcpy(group_of_mat, c->group_of_mat.data(), sizeof(int) * c->n_mats);
+  if (order_in_group) memcpy(order_in_group, c->order_in_group.data(), sizeof(int) * c->n_mats);
+  return PRM_OK;
+}
+
+static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepScalars s,
+                         cudaStream_t stream) {
+  const size_t e = c->check_mode ? 4 : 2;
+  const int64_t rc = g.rp * g.cp, rr = g.rp * g.rp;
+  float* fro = (float*)(c->ws + c->off_fro);
+  float* alpha = (float*)(c->ws + c->off_alpha);
+  int* status = (int*)(c->ws + c->off_status);
+  for (int done = 0; done < g.count; done += g.ns_batch) {
+    const int nb = std::min(g.ns_batch, g.count - done);
+    char* base = c->ws + c->off_ns;
+    char* X[2] = {base, base + e * rc * nb};
+    char* XT[2] = {base + 2 * e * rc * nb, base + 3 * e * rc * nb};
+    char* A = base + 4 * e * rc * nb;
+    char* B = A + e * rr * nb;
+    const int first = g.first + done;
+    cudaError_t ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, c->check_mode, X[0], XT[0],
+                                       fro, alpha, stream, &c->launches);
+    if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("pre-pass: ") + cudaGetErrorString(ce));
+    auto gemm = [&](const GemmProblem& pb, const Epilogue& ep) -> cudaError_t {
+      return c->check_mode ? launch_gemm_simt(pb, ep, stream, &c->launches)
+                           : launch_gemm_tc(c->tc, pb, ep, status, stream, &c->launches);
+    };
+    int cur = 0;
+    for (int it = 0; it < kNsIters; ++it) {
+      // A = X X^T (times alpha^2 in the first iteration)
+      GemmProblem pa;
+      pa.P = X[cur]; pa.Q = X[cur]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
+      pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
+      Epilogue ea;
+      ea.dst = A; ea.ld_dst = g.rp; ea.bs_dst = rr;
+      ea.dst_t = A; ea.ld_dst_t = g.rp; ea.bs_dst_t = rr;
+      if (it == 0) { ea.alpha = alpha; ea.alpha_pow = 2; }
+      if ((ce = gemm(pa, ea)) != cudaSuccess) break;
+      // B = b A + c A^2
+      GemmProblem pp;
+      pp.P = A; pp.Q = A; pp.Mp = g.rp; pp.Np = g.rp; pp.Kp = g.rp;
+      pp.bs_P = rr; pp.bs_Q = rr; pp.batch = nb; pp.symmetric = 1;
+      Epilogue eb;
+      eb.k_acc = kNsC; eb.k_aux = kNsB; eb.aux = A; eb.ld_aux = g.rp; eb.bs_aux = rr;
+      eb.dst = B; eb.ld_dst = g.rp; eb.bs_dst = rr;
+      eb.dst_t = B; eb.ld_dst_t = g.rp; eb.bs_dst_t = rr;
+      if ((ce = gemm(pp, eb)) != cudaSuccess) break;
+      // X <- a X + B X (times alpha in the first iteration); last iteration
+      // goes straight into the parameters.
+      GemmProblem pu;
+      pu.P = B; pu.Q = XT[cur]; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
+      pu.bs_P = rr; pu.bs_Q = rc; pu.batch = nb; pu.symmetric = 0;
+      Epilogue eu;
+      eu.k_acc = 1.f; eu.k_aux = kNsA; eu.aux = X[cur]; eu.ld_aux = g.cp; eu.bs_aux = rc;
+      if (it == 0) { eu.alpha = alpha; eu.alpha_pow = 1; }
+      if (it + 1 < kNsIters) {
+        eu.dst = X[cur ^ 1]; eu.ld_dst = g.cp; eu.bs_dst = rc;
+        eu.dst_t = XT[cur ^ 1]; eu.ld_dst_t = g.rp; eu.bs_dst_t = rc;
+      } else {
+        eu.kind = 1; eu.tables = t; eu.first = first;
+        eu.rows = (int)g.rows; eu.cols = (int)g.cols; eu.tall = g.tall ? 1 : 0;
+        eu.io_fp32 = c->io_fp32; eu.decay = s.decay; eu.lr_s = s.lr_s;
+      }
+      if ((ce = gemm(pu, eu)) != cudaSuccess) break;
+      cur ^= 1;
+    }
+    if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("NS5 product: ") + cudaGetErrorString(ce));
+  }
+  return PRM_OK;
+}
+
+static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
+                     const void* const* grads_host, float* const* momentum, int64_t step_idx,
+                     cudaStream_t stream) {
+  if (!c) return PRM_ERR_ARG;
+  if (!params || !grads_dev || !momentum) return fail(c, PRM_ERR_ARG, "prm_step: NULL pointer array");
+  if (step_idx < 0) return fail(c, PRM_ERR_ARG, "prm_step: negative step index");
+  if (!c->ws) return fail(c, PRM_ERR_WORKSPACE, "prm_step: no workspace attached");
+  bool changed = !c->tables_uploaded;
+  const int n = c->n_mats;
+  for (int i = 0; i < n; ++i) {
+    if (!params[i] || !grads_dev[i] || !momentum[i]) return fail(c, PRM_ERR_ARG, "prm_step: NULL matrix pointer");
+    if ((((uintptr_t)params[i] | (uintptr_t)grads_dev[i] | (uintptr_t)momentum[i]) & 15) != 0)
+      return fail(c, PRM_ERR_ALIGN, "prm_step: matrix pointer not 16-byte aligned");
+    const int slot = c->slot_of_mat[i];
+    void* want[3] = {params[i], grads_dev[i], (void*)momentum[i]};
+    for (int k = 0; k < 3; ++k) {
+      if (c->host_tables[(size_t)k * n + slot] != want[k]) { c->host_tables[(size_t)k * n + slot] = want[k]; changed = true; }
+    }
+  }
+  cudaError_t ce;
+  if (changed) {
+    // Pageable source: the runtime stages the bytes before returning.
+    ce = cudaMemcpyAsync(c->ws + c->off_tables, c->host_tables.data(), (size_t)3 * n * sizeof(void*),
+                         cudaMemcpyHostToDevice, stream);
+    if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("pointer tables: ") + cudaGetErrorString(ce));
+    c->tables_uploaded = true;
+  }
+  if (grads_host) {
+    const size_t esz = c->io_fp32 ? 4 : 2;
+    for (int i = 0; i < n; ++i) {
+      if (!grads_host[i]) return fail(c, PRM_ERR_ARG, "prm_step_h2d: NULL host gradient pointer");
+      ce = cudaMemcpyAsync(grads_dev[i], grads_host[i], esz * (size_t)c->shapes[2 * i] * (size_t)c->shapes[2 * i + 1],
+                           cudaMemcpyHostToDevice, stream);
+      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("gradient copy: ") + cudaGetErrorString(ce));
+    }
+  }
+  PtrTables t;
+  void** tb = (void**)(c->ws + c->off_tables);
+  t.params = tb;
+  t.grads = (const void**)(tb + n);
+  t.momentum = (float**)(tb + 2 * n);
+  const bool refresh = (step_idx % c->K) == 0;
+  for (const Group& g : c->groups) {
+    StepScalars s;
+    s.beta = c->beta; s.omb = 1.f - c->beta; s.nesterov = c->nesterov;
+    s.decay = 1.f - c->lr * c->wd;
+    s.lr_s = c->lr * shape_scale(c->scale_mode, g.rows, g.cols);
+    s.gamma = c->gamma; s.eps_row = c->eps_row; s.eps_ns = c->eps_ns;
+    if (refresh) {
+      int rc = refresh_group(c, g, t, s, stream);
+      if (rc != PRM_OK) return rc;
+    } else {
+      ce = launch_rowstep(t, g, s, c->io_fp32, (float*)(c->ws + g.tall_scratch_off),
+                          (float*)(c->ws + g.tall_nu_off), stream, &c->launches);
+      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("row step: ") + cudaGetErrorString(ce));
+    }
+  }
+  return PRM_OK;
+}
+
+extern "C" int prm_step(prm_ctx* c, void* const* params, const void* const* grads,
+                        float* const* momentum, int64_t step_idx, void* cuda_stream) {
+  return step_impl(c, params, (void* const*)grads, nullptr, momentum, step_idx, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int prm_step_h2d(prm_ctx* c, void* const* params, void* const* grads_dev,
+                            const void* const* grads_host, float* const* momentum,
+                            int64_t step_idx, void* cuda_stream) {
+  if (c && !grads_host) return fail(c, PRM_ERR_ARG, "prm_step_h2d: NULL host gradient array");
+  return step_impl(c, params, grads_dev, grads_host, momentum, step_idx, (cudaStream_t)cuda_stream);
+}
+
+extern "C" int prm_status(prm_ctx* c) {
+  if (!c) return PRM_ERR_ARG;
+  if (!c->ws) return fail(c, PRM_ERR_WORKSPACE, "prm_status: no workspace attached");
+  cudaError_t ce = cudaDeviceSynchronize();
+  int word = 0;
+  if (ce == cudaSuccess) ce = cudaMemcpy(&word, c->ws + c->off_status, sizeof(int), cudaMemcpyDeviceToHost);
+  if (ce == cudaSuccess && word != 0) ce = cudaMemset(c->ws + c->off_status, 0, sizeof(int));
+  if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("prm_status: ") + cudaGetErrorString(ce));
+  if (word & kStatusTimeout) return fail(c, PRM_ERR_DEVICE_TIMEOUT, "a device-side wait gave up");
+  return PRM_OK;
+}
+
+extern "C" const char* prm_last_error(const prm_ctx* c) { return c ? c->err.c_str() : g_create_err.c_str(); }
+
+extern "C" int64_t prm_launch_count(const prm_ctx* c) { return c ? c->launches : 0; }
+
+extern "C" int prm_destroy(prm_ctx* c) {
+  if (!c) return PRM_ERR_ARG;
+  if (c->tc) tc_destroy(c->tc);
+  delete c;
+  return PRM_OK;
+}

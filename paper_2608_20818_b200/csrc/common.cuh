@@ -1,0 +1,156 @@
+// Shared device helpers and host-side plan structures of the prm library.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/prm.h"
+
+namespace prm {
+
+// ---------------------------------------------------------------- constants
+// Newton-Schulz coefficients and iteration count (paper, appendix "Optimizer
+// and Training Hyperparameters").
+constexpr float kNsA = 3.4445f;
+constexpr float kNsB = -4.7750f;
+constexpr float kNsC = 2.0315f;
+constexpr int kNsIters = 5;
+
+// NS5 operands live in the workspace padded to multiples of kPad in both
+// dimensions; the padding is zero and stays zero through the recurrence.
+constexpr int kPad = 256;
+
+// Tall row-step: rows per column-partial block.
+constexpr int kTallRows = 128;
+// Tall row-step and pre-pass: columns per CTA.
+constexpr int kTallCols = 256;
+
+// Device status word values (bit flags).
+constexpr int kStatusTimeout = 1;
+
+// ------------------------------------------------------------- I/O helpers
+struct alignas(16) bf16x8 {
+  __nv_bfloat162 v[4];
+};
+
+// Load 8 consecutive elements as fp32.
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&out)[8]) {
+  bf16x8 raw = *reinterpret_cast<const bf16x8*>(p);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 f = __bfloat1622float2(raw.v[i]);
+    out[2 * i] = f.x;
+    out[2 * i + 1] = f.y;
+  }
+}
+__device__ __forceinline__ void load8(const float* p, float (&out)[8]) {
+  float4 a = *reinterpret_cast<const float4*>(p);
+  float4 b = *reinterpret_cast<const float4*>(p + 4);
+  out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+  out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+}
+// Streaming variants for data that is read exactly once.
+__device__ __forceinline__ void load8_stream(const __nv_bfloat16* p, float (&out)[8]) {
+  int4 r = __ldcs(reinterpret_cast<const int4*>(p));
+  bf16x8 raw = *reinterpret_cast<bf16x8*>(&r);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float2 f = __bfloat1622float2(raw.v[i]);
+    out[2 * i] = f.x;
+    out[2 * i + 1] = f.y;
+  }
+}
+__device__ __forceinline__ void load8_stream(const float* p, float (&out)[8]) {
+  float4 a = __ldcs(reinterpret_cast<const float4*>(p));
+  float4 b = __ldcs(reinterpret_cast<const float4*>(p + 4));
+  out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+  out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+}
+// Eight elements kept in their storage format (registers), converted on use.
+template <typename T> struct Raw8;
+template <> struct Raw8<__nv_bfloat16> {
+  int4 r;
+  __device__ __forceinline__ void load_stream(const __nv_bfloat16* p) { r = __ldcs(reinterpret_cast<const int4*>(p)); }
+  __device__ __forceinline__ void get(float (&out)[8]) const {
+    const __nv_bfloat162* v = reinterpret_cast<const __nv_bfloat162*>(&r);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float2 f = __bfloat1622float2(v[i]);
+      out[2 * i] = f.x;
+      out[2 * i + 1] = f.y;
+    }
+  }
+};
+template <> struct Raw8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load_stream(const float* p) {
+    a = __ldcs(reinterpret_cast<const float4*>(p));
+    b = __ldcs(reinterpret_cast<const float4*>(p + 4));
+  }
+  __device__ __forceinline__ void get(float (&out)[8]) const {
+    out[0] = a.x; out[1] = a.y; out[2] = a.z; out[3] = a.w;
+    out[4] = b.x; out[5] = b.y; out[6] = b.z; out[7] = b.w;
+  }
+};
+
+// Store 8 consecutive elements (fp32 -> bf16 is round-to-nearest-even).
+__device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&in)[8]) {
+  bf16x8 raw;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) raw.v[i] = __floats2bfloat162_rn(in[2 * i], in[2 * i + 1]);
+  *reinterpret_cast<bf16x8*>(p) = raw;
+}
+__device__ __forceinline__ void store8(float* p, const float (&in)[8]) {
+  *reinterpret_cast<float4*>(p) = make_float4(in[0], in[1], in[2], in[3]);
+  *reinterpret_cast<float4*>(p + 4) = make_float4(in[4], in[5], in[6], in[7]);
+}
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ void from_f32(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
+__device__ __forceinline__ void from_f32(float* p, float x) { *p = x; }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ------------------------------------------------------------ host structs
+// Per-step scalar hyper-parameters handed to kernels by value.
+struct StepScalars {
+  float beta;      // momentum coefficient
+  float omb;       // 1 - beta
+  int nesterov;
+  float decay;     // 1 - lr*wd
+  float lr_s;      // lr * s(W) for the group
+  float gamma;
+  float eps_row;
+  float eps_ns;
+};
+
+// Device pointer tables, ordered by (group, order in group).
+struct PtrTables {
+  void** params;          // [n_mats]
+  const void** grads;     // [n_mats]
+  float** momentum;       // [n_mats]
+};
+
+struct Group {
+  int64_t rows = 0, cols = 0;   // stored shape
+  int count = 0;                // matrices in the group
+  int first = 0;                // index of the group's first matrix in the grouped order
+  bool tall = false;
+  int64_t r = 0, c = 0;         // oriented shape, r <= c
+  int64_t rp = 0, cp = 0;       // padded oriented shape (NS5 workspace)
+  int ns_batch = 1;             // matrices refreshed per sub-batch
+  size_t tall_scratch_off = 0;  // byte offset of column partials (tall groups)
+  size_t tall_nu_off = 0;       // byte offset of column norms (tall groups)
+};
+
+inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+}  // namespace prm

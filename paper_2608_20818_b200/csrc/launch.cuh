@@ -1,0 +1,71 @@
+// Host-side launch interfaces between the scheduler (api.cu) and the kernels.
+#pragma once
+
+#include "common.cuh"
+
+namespace prm {
+
+// Epilogue of every NS5 product D[i,j] = sum_k P[i,k]*Q[j,k] (both operands
+// row-major with k contiguous).  With f = alpha[b]^alpha_pow (1 if alpha is
+// null) and v = f*(k_acc*D[i,j] + k_aux*aux[i,j]):
+//   kind 0: dst[i,j] = v; if dst_t is set, dst_t[j,i] = v as well (for the
+//           symmetric products this is the mirror write of the other
+//           triangle, for the X update it is the transposed copy of X).
+//   kind 1: parameter update W = decay*W - lr_s*v at the stored position of
+//           oriented element (i,j) (Eq. periodic-direction, rho_t = 1).
+struct Epilogue {
+  int kind = 0;
+  float k_acc = 1.f, k_aux = 0.f;
+  const float* alpha = nullptr;   // [batch] 1/(||U||_F + eps_ns)
+  int alpha_pow = 0;
+  const void* aux = nullptr;      // [batch][Mp][ld_aux]
+  int64_t ld_aux = 0, bs_aux = 0;
+  void* dst = nullptr;            // [batch][Mp][ld_dst]
+  int64_t ld_dst = 0, bs_dst = 0;
+  void* dst_t = nullptr;          // [batch][Np][ld_dst_t]
+  int64_t ld_dst_t = 0, bs_dst_t = 0;
+  // kind 1
+  PtrTables tables = {};
+  int first = 0;                  // table index of the sub-batch's first matrix
+  int rows = 0, cols = 0;         // stored shape
+  int tall = 0;
+  int io_fp32 = 0;
+  float decay = 1.f, lr_s = 0.f;
+};
+
+// One batched product.  P: [batch][Mp][Kp], Q: [batch][Np][Kp]; Mp, Np, Kp
+// are multiples of kPad.  symmetric != 0: P == Q and only tiles of the lower
+// triangle are computed, the rest is filled by the mirror write.
+struct GemmProblem {
+  const void* P = nullptr;
+  const void* Q = nullptr;
+  int64_t Mp = 0, Np = 0, Kp = 0;
+  int64_t bs_P = 0, bs_Q = 0;     // batch strides in elements
+  int batch = 1;
+  int symmetric = 0;
+};
+
+cudaError_t launch_rowstep(const PtrTables& t, const Group& g, const StepScalars& s, int io_fp32,
+                           float* tall_partial, float* tall_nu, cudaStream_t stream,
+                           int64_t* launches);
+
+// Momentum update + direction input written to the NS5 workspace in both
+// orientations, with per-CTA partial sums of squares, then alpha per matrix.
+// x_fp32: workspace element type (1: fp32 check mode, 0: bf16).
+cudaError_t launch_ns_prepass(const PtrTables& t, const Group& g, int first, int batch,
+                              const StepScalars& s, int io_fp32, int x_fp32, void* X, void* XT,
+                              float* fro_partial, float* alpha, cudaStream_t stream,
+                              int64_t* launches);
+
+// fp32 CUDA-core product (check mode).
+cudaError_t launch_gemm_simt(const GemmProblem& pb, const Epilogue& ep, cudaStream_t stream,
+                             int64_t* launches);
+
+// bf16 tensor-core product (tcgen05, TMEM accumulators, TMA-fed tiles).
+struct TcContext;
+cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue& ep, int* status,
+                           cudaStream_t stream, int64_t* launches);
+TcContext* tc_create(std::string* err);
+void tc_destroy(TcContext* tc);
+
+}  // namespace prm

@@ -1,0 +1,150 @@
+// NS5 pre-pass: the refresh step's only read of gradients and momentum.
+//
+// For every matrix of a sub-batch it updates the momentum in place
+// (Algorithm 1 line 2), forms the direction input U, and writes U - unscaled -
+// into the NS5 workspace in both orientations: X (r x c, the oriented matrix
+// of Section 3.1) and XT (c x r).  All NS5 products then read both operands
+// with the contraction index contiguous.  The Frobenius norm of U is reduced
+// alongside (per-CTA partials, then one fixed-order sum per matrix) and
+// enters the recurrence as alpha = 1/(||U||_F + eps_ns) in the first
+// iteration's epilogues, so the normalisation costs no extra pass.
+//
+// The workspace copies are zero-padded to multiples of kPad; zero rows and
+// columns stay zero under X -> aX + (bA + cA^2)X.
+#include "launch.cuh"
+
+namespace prm {
+
+constexpr int kPreTile = 64;
+constexpr int kPreThreads = 256;
+
+template <typename IO, typename XT_, bool VEC>
+__global__ void __launch_bounds__(kPreThreads)
+ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
+                  XT_* __restrict__ straight, int64_t ld_s, int64_t bs_s,
+                  XT_* __restrict__ transposed, int64_t ld_t, int64_t bs_t,
+                  float* __restrict__ fro_partial) {
+  __shared__ float tile[kPreTile][kPreTile + 1];
+  __shared__ float warp_part[kPreThreads / 32];
+  const int b = blockIdx.z;
+  const IO* __restrict__ g = reinterpret_cast<const IO*>(t.grads[first + b]);
+  float* __restrict__ m = t.momentum[first + b];
+  XT_* __restrict__ ds = straight + (int64_t)b * bs_s;
+  XT_* __restrict__ dt = transposed + (int64_t)b * bs_t;
+  const int r0 = blockIdx.y * kPreTile, c0 = blockIdx.x * kPreTile;
+  const int tx = threadIdx.x & 7, ty = threadIdx.x >> 3;   // 8 column vectors x 32 rows
+  float acc = 0.f;
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const int lr = ty + 32 * half;
+    const int row = r0 + lr, col = c0 + tx * 8;
+    float u[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) u[e] = 0.f;
+    if (row < rows) {
+      const int64_t off = (int64_t)row * cols + col;
+      if (VEC) {
+        if (col < cols) {
+          float gv[8], mv[8];
+          load8_stream(g + off, gv);
+          load8_stream(m + off, mv);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+            const float mn = s.beta * mv[e] + s.omb * gv[e];
+            mv[e] = mn;
+            u[e] = s.nesterov ? s.beta * mn + s.omb * gv[e] : mn;
+          }
+          store8(m + off, mv);
+        }
+      } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (col + e < cols) {
+            const float gv = to_f32(g[off + e]);
+            const float mn = s.beta * m[off + e] + s.omb * gv;
+            m[off + e] = mn;
+            u[e] = s.nesterov ? s.beta * mn + s.omb * gv : mn;
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      acc += u[e] * u[e];
+      tile[lr][tx * 8 + e] = u[e];
+    }
+    store8(ds + (int64_t)row * ld_s + col, u);   // padded extent: always in range
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kPreThreads / 32; ++w) tot += warp_part[w];
+    fro_partial[((int64_t)b * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x] = tot;
+  }
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const int lc = ty + 32 * half;            // column of the tile = row of the transposed copy
+    float u[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) u[e] = tile[tx * 8 + e][lc];
+    store8(dt + (int64_t)(c0 + lc) * ld_t + r0 + tx * 8, u);
+  }
+}
+
+// alpha[b] = 1/(sqrt(sum of partials) + eps_ns); one CTA per matrix, fixed
+// summation order.
+__global__ void __launch_bounds__(kPreThreads)
+ns_alpha_kernel(const float* __restrict__ fro_partial, int nparts, float eps_ns,
+                float* __restrict__ alpha) {
+  __shared__ float part[kPreThreads];
+  const float* src = fro_partial + (int64_t)blockIdx.x * nparts;
+  float acc = 0.f;
+  for (int i = threadIdx.x; i < nparts; i += kPreThreads) acc += src[i];
+  part[threadIdx.x] = acc;
+  __syncthreads();
+  for (int w = kPreThreads / 2; w > 0; w >>= 1) {
+    if (threadIdx.x < w) part[threadIdx.x] += part[threadIdx.x + w];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) alpha[blockIdx.x] = 1.f / (sqrtf(part[0]) + eps_ns);
+}
+
+template <typename IO, typename XT_>
+static cudaError_t prepass_inst(const PtrTables& t, const Group& g, int first, int batch,
+                                const StepScalars& s, XT_* X, XT_* XT, float* fro_partial,
+                                float* alpha, cudaStream_t stream) {
+  // Stored extent padded: wide -> (rp, cp), tall -> (cp, rp).
+  const int64_t prow = g.tall ? g.cp : g.rp, pcol = g.tall ? g.rp : g.cp;
+  XT_* straight = g.tall ? XT : X;
+  XT_* transposed = g.tall ? X : XT;
+  const int64_t bs = g.rp * g.cp;
+  dim3 grid((unsigned)(pcol / kPreTile), (unsigned)(prow / kPreTile), (unsigned)batch);
+  if (grid.y > 65535 || grid.z > 65535) return cudaErrorInvalidValue;
+  const bool vec = (g.cols % 8 == 0);
+  if (vec)
+    ns_prepass_kernel<IO, XT_, true><<<grid, kPreThreads, 0, stream>>>(
+        t, first, (int)g.rows, (int)g.cols, s, straight, pcol, bs, transposed, prow, bs, fro_partial);
+  else
+    ns_prepass_kernel<IO, XT_, false><<<grid, kPreThreads, 0, stream>>>(
+        t, first, (int)g.rows, (int)g.cols, s, straight, pcol, bs, transposed, prow, bs, fro_partial);
+  ns_alpha_kernel<<<batch, kPreThreads, 0, stream>>>(fro_partial, (int)(grid.x * grid.y), s.eps_ns, alpha);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_ns_prepass(const PtrTables& t, const Group& g, int first, int batch,
+                              const StepScalars& s, int io_fp32, int x_fp32, void* X, void* XT,
+                              float* fro_partial, float* alpha, cudaStream_t stream,
+                              int64_t* launches) {
+  *launches += 2;
+  if (io_fp32) {
+    if (x_fp32) return prepass_inst<float, float>(t, g, first, batch, s, (float*)X, (float*)XT, fro_partial, alpha, stream);
+    return prepass_inst<float, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, (__nv_bfloat16*)XT, fro_partial, alpha, stream);
+  }
+  if (x_fp32) return prepass_inst<__nv_bfloat16, float>(t, g, first, batch, s, (float*)X, (float*)XT, fro_partial, alpha, stream);
+  return prepass_inst<__nv_bfloat16, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, (__nv_bfloat16*)XT, fro_partial, alpha, stream);
+}
+
+}  // namespace prm

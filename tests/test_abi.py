@@ -1,0 +1,97 @@
+"""CPU-side checks of the C ABI: the library loads, exports what the header
+declares, validates arguments, and its plan matches the oracle bit for bit."""
+
+import os
+import re
+
+import pytest
+
+from oracle import prm_oracle as O
+from paper_2608_20818_b200 import binding as B
+from paper_2608_20818_b200 import build as build_mod
+from paper_2608_20818_b200.workloads import workload
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_mod.build()
+
+
+def test_exports_match_header():
+    hdr = open(os.path.join(ROOT, "include", "prm.h")).read()
+    declared = set(re.findall(r"PRM_API\s+[\w\s\*]+?\b(prm_\w+)\s*\(", hdr))
+    assert declared == set(B.EXPORTS)
+    L = B.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_option_constants_match_header():
+    hdr = open(os.path.join(ROOT, "include", "prm.h")).read()
+    for name, val in re.findall(r"#define\s+(PRM_(?:OPT|ERR)_\w+|PRM_OK)\s+(-?\d+)", hdr):
+        assert getattr(B, name) == int(val), name
+
+
+@pytest.mark.parametrize("cfg_id", [1, 2, 3, 4, 5])
+def test_plan_matches_oracle(cfg_id):
+    wl = workload(cfg_id)
+    h = B.prm_create(wl.shapes, wl.K, wl.beta, wl.nesterov, wl.lr, wl.wd)
+    g_ref, o_ref, gs = O.group_by_shape(wl.shapes)
+    for t in range(0, 2 * wl.K + 1):
+        refresh, n_groups, g, o = B.prm_plan(h, t, len(wl.shapes))
+        assert refresh == O.is_refresh(t, wl.K)
+        assert n_groups == len(gs) and g == g_ref and o == o_ref
+    assert B.prm_workspace_bytes(h) > 0
+    B.prm_destroy(h)
+
+
+def test_plan_mixed_shapes_and_k1():
+    shapes = [(2, 6), (2, 2), (8, 2), (2, 8), (2, 6), (8, 2), (2, 2)]
+    h = B.prm_create(shapes, 1, 0.9, False, 1e-3, 0.0)
+    refresh, n_groups, g, o = B.prm_plan(h, 7, len(shapes))
+    assert refresh and n_groups == 4
+    assert g == [0, 1, 2, 3, 0, 2, 1] and o == [0, 0, 0, 0, 1, 1, 1]
+    B.prm_destroy(h)
+
+
+def test_argument_errors():
+    with pytest.raises(B.PrmError) as e:
+        B.prm_create([(4, 4)], 0, 0.95, False, 1e-3, 0.0)
+    assert e.value.code == B.PRM_ERR_ARG
+    with pytest.raises(B.PrmError) as e:
+        B.prm_create([(4, 0)], 2, 0.95, False, 1e-3, 0.0)
+    assert e.value.code == B.PRM_ERR_SHAPE
+    with pytest.raises(B.PrmError) as e:
+        B.prm_create([], 2, 0.95, False, 1e-3, 0.0)
+    assert e.value.code == B.PRM_ERR_ARG
+    with pytest.raises(B.PrmError) as e:
+        B.prm_create([(4, 4)], 2, 1.5, False, 1e-3, 0.0)
+    assert e.value.code == B.PRM_ERR_ARG
+    h = B.prm_create([(4, 4)], 2, 0.95, False, 1e-3, 0.0)
+    with pytest.raises(B.PrmError) as e:
+        B.prm_set_option(h, 999, 1.0)
+    assert e.value.code == B.PRM_ERR_ARG
+    with pytest.raises(B.PrmError) as e:
+        B.prm_set_option(h, B.PRM_OPT_SCALE_MODE, 5)
+    assert e.value.code == B.PRM_ERR_ARG
+    # a step without a workspace is refused before any device work
+    import ctypes
+    arr = (ctypes.c_void_p * 1)(16)
+    with pytest.raises(B.PrmError) as e:
+        B.prm_step(h, arr, arr, arr, 0)
+    assert e.value.code == B.PRM_ERR_WORKSPACE
+    B.prm_destroy(h)
+
+
+def test_workspace_scales_with_options():
+    shapes = [(512, 1024)] * 4
+    h = B.prm_create(shapes, 2, 0.95, False, 1e-3, 0.0)
+    fast = B.prm_workspace_bytes(h)
+    B.prm_set_option(h, B.PRM_OPT_CHECK_MODE, 1)
+    check = B.prm_workspace_bytes(h)
+    assert check > fast
+    B.prm_set_option(h, B.PRM_OPT_NS_WORKSPACE_BYTES, 1)
+    assert B.prm_workspace_bytes(h) < check
+    B.prm_destroy(h)

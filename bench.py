@@ -1,0 +1,371 @@
+#!/usr/bin/env python
+"""Benchmark of the Periodic Row-wise Muon optimizer step on B200.
+
+    python bench.py [--gpus N] [--steps S] [--warmup W] [--config 4] [--K 5]
+    python bench.py --impl reference ...      # the fp64 CPU oracle on the host cores
+
+One "step" is one prm_step over the whole shape set (a refresh when
+step_idx mod K == 0, a row step otherwise).  The line printed by rank 0 holds
+the amortised optimizer ms/step at K, with per-branch times, the row-step
+GB/s, the NS5 TFLOP/s, a roofline entry for the dominant kernel and the
+oracle's CPU baseline.
+"""
+
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2608_20818_b200.workloads import make_grad, make_momentum, make_param, workload  # noqa: E402
+
+METRIC = "amortised optimizer ms/step at K"
+NOMINAL_HBM_GBS = 8000.0       # nominal figure the targets are quoted against
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+# ----------------------------------------------------------------- accounting
+def ns5_flops(shapes):
+    """(executed with symmetry, paper model) flop of one refresh."""
+    ex = mo = 0
+    for (m, n) in shapes:
+        r, c = min(m, n), max(m, n)
+        ex += 15 * r * r * c + 5 * r ** 3
+        mo += 20 * r * r * c + 10 * r ** 3
+    return ex, mo
+
+
+def elements(shapes):
+    return sum(m * n for (m, n) in shapes)
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.Q}",
+                                       "--format=csv,noheader,nounits", "-lms", "200"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------- CPU oracle
+def oracle_sample(wl, K, budget_s=10.0):
+    """Times the fp64 oracle on a bounded sample of the workload and scales it
+    to the whole shape set: one refresh and one row step on a square r x r
+    matrix (r <= d chosen so the refresh fits the time budget), scaled by the
+    paper's flop model (refresh) and by element count (row step)."""
+    import numpy as np
+    from oracle import prm_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    cfg = O.OracleConfig(K=K, beta=wl.beta, nesterov=wl.nesterov, lr=wl.lr, wd=wl.wd, gamma=wl.gamma)
+    rng = np.random.default_rng(20818)
+    d = max(min(m, n) for (m, n) in wl.shapes)
+
+    def one(r, t):
+        W = rng.standard_normal((r, r)) * 0.02
+        G = rng.standard_normal((r, r)) * wl.grad_std
+        M = rng.standard_normal((r, r)) * wl.grad_std
+        t0 = time.perf_counter()
+        O.step_matrix(W, G, M, t, cfg)
+        return time.perf_counter() - t0
+
+    probe = min(d, 512)
+    one(probe, 0)
+    rate = 30.0 * probe ** 3 / max(one(probe, 0), 1e-6)          # flop/s of the refresh at probe size
+    r = int(min(d, max(probe, (budget_s * rate / 30.0) ** (1.0 / 3.0)))) // 64 * 64
+    r = max(r, min(d, 64))
+    t_ref = one(r, 0)
+    t_row = one(r, 1) if K > 1 else 0.0
+    _, model = ns5_flops(wl.shapes)
+    ref_ms = 1e3 * t_ref * model / (30.0 * r ** 3)
+    row_ms = 1e3 * t_row * elements(wl.shapes) / float(r * r)
+    amort = (ref_ms + (K - 1) * row_ms) / K
+    sample = (f"one refresh and one row step of the oracle on a {r}x{r} matrix "
+              f"({t_ref:.2f} s, {t_row:.3f} s), scaled to the shape set by the 20r^2c+10r^3 flop model "
+              f"(refresh) and by element count (row step)")
+    return {"value": amort, "unit": "ms/step", "cores": cores, "kind": "oracle", "sample": sample,
+            "refresh_ms": ref_ms, "row_step_ms": row_ms}
+
+
+def run_reference(args, wl, K):
+    """The reference arm: the oracle as it stands on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    base = None
+    per = max(2.0, min(10.0, 120.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup + args.steps):
+        base = oracle_sample(wl, K, budget_s=per)
+        if i >= args.warmup:
+            vals.append(base["value"])
+    v = sum(vals) / len(vals)
+    base["value"] = v
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": "ms/step", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": v, "higher_is_better": False,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "K": K, "matrices": len(wl.shapes)},
+            "cpu_baseline": base,
+            "e2e": {"value": v, "unit": "ms/step", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------- GPU arm
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="prm", choices=["prm", "reference"])
+    ap.add_argument("--config", type=int, default=4, help="benchmark configuration 2..5 (default 4: 9B-class)")
+    ap.add_argument("--blocks", type=int, default=None, help="override the number of transformer blocks")
+    ap.add_argument("--K", type=int, default=None)
+    ap.add_argument("--check-mode", action="store_true", help="NS5 in fp32 on CUDA cores")
+    ap.add_argument("--first-step", type=int, default=None, help="step index of the first warm-up step")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+
+    wl = workload(args.config, args.blocks)
+    K = args.K or wl.K
+    if args.steps is None:
+        args.steps = 2 * K
+    if args.warmup is None:
+        args.warmup = max(3, K)
+    if args.impl == "reference":
+        run_reference(args, wl, K)
+        return
+
+    from paper_2608_20818_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = world > 1
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if dist:
+        import torch.distributed as td
+        td.init_process_group("nccl", device_id=dev)
+
+    n = len(wl.shapes)
+    io_bytes = 4 if wl.io_dtype == "fp32" else 2
+    opt = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
+                                io_dtype=wl.io_dtype, check_mode=args.check_mode, device=dev)
+    params = [make_param(wl, i, dev) for i in range(n)]
+    moms = [make_momentum(wl, i, dev) for i in range(n)]
+    # One gradient set per matrix kind and step parity keeps generation cheap;
+    # every matrix still owns its own gradient buffer in HBM.
+    grads = [make_grad(wl, i, 0, dev) for i in range(n)]
+    torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream(dev)
+    t_first = (K - (args.warmup % K)) % K            # so that the first timed step is a refresh
+    if args.first_step is not None:
+        t_first = args.first_step
+    step_idx = t_first
+
+    def barrier():
+        if dist:
+            td.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        opt.step(params, grads, moms, step_idx)
+        step_idx += 1
+    barrier()
+    assert opt.status() == B.PRM_OK, "device status after warm-up"
+
+    launches0 = opt.launch_count()
+    opt.profile(True)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    kinds = []
+    barrier()
+    ev[0].record(stream)
+    for k in range(args.steps):
+        kinds.append(opt.plan(step_idx)[0])
+        opt.step(params, grads, moms, step_idx)
+        ev[k + 1].record(stream)
+        step_idx += 1
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    prof = opt.profile_read()
+    opt.profile(False)
+    launches = opt.launch_count() - launches0
+    assert opt.status() == B.PRM_OK, "device status after the timed region"
+
+    per_step = [ev[k].elapsed_time(ev[k + 1]) for k in range(args.steps)]
+    total_ms = ev[0].elapsed_time(ev[args.steps])
+    ref_ms = [t for t, r in zip(per_step, kinds) if r]
+    row_ms = [t for t, r in zip(per_step, kinds) if not r]
+    stats = torch.tensor([total_ms, sum(ref_ms) / max(1, len(ref_ms)), sum(row_ms) / max(1, len(row_ms))],
+                         dtype=torch.float64, device=dev)
+    if dist:
+        td.all_reduce(stats, op=td.ReduceOp.MAX)
+    total_ms, mean_ref, mean_row = [float(x) for x in stats.cpu()]
+
+    # ---------------------------------------------------------- e2e (host grads)
+    e2e = None
+    if not args.no_e2e:
+        block = 5 if wl.config_id != 1 else 1
+        host = [torch.empty(wl.shapes[i], dtype=grads[i].dtype).pin_memory() for i in range(min(block, n))]
+        for i, h in enumerate(host):
+            h.copy_(grads[i])
+        grads_host = [host[i % block] for i in range(n)]
+        readback = torch.empty(1024, dtype=params[0].dtype).pin_memory()
+        h2d = sum(m * nn for (m, nn) in wl.shapes) * io_bytes
+        d2h = readback.numel() * readback.element_size() + 4
+        e_steps = args.steps
+        barrier()
+        t0 = torch.cuda.Event(enable_timing=True)
+        t1 = torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for k in range(e_steps):
+            opt.step_h2d(params, grads, grads_host, moms, step_idx)
+            readback.copy_(params[0].view(-1)[:1024], non_blocking=True)
+            stream.synchronize()
+            assert opt.status() == B.PRM_OK
+            step_idx += 1
+        t1.record(stream)
+        barrier()
+        e_ms = torch.tensor([t0.elapsed_time(t1) / e_steps], dtype=torch.float64, device=dev)
+        if dist:
+            td.all_reduce(e_ms, op=td.ReduceOp.MAX)
+        e2e = {"value": float(e_ms.cpu()) / world, "unit": "ms/step", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h,
+               "note": "gradients copied every step from pinned host memory (one block's gradients, reused "
+                       "for every block) through prm_step_h2d; 2 KB of parameters and the status word read back"}
+
+    if rank != 0:
+        if dist:
+            td.destroy_process_group()
+        return
+
+    pk = peaks()
+    amort = (mean_ref + (K - 1) * mean_row) / K if (ref_ms and (row_ms or K == 1)) else total_ms / args.steps
+    n_ref, n_row = len(ref_ms), len(row_ms)
+    ex, mo = ns5_flops(wl.shapes)
+    el = elements(wl.shapes)
+    row_bytes = el * (3 * io_bytes + 8)   # g and p read, p write (I/O dtype), m read and write (fp32)
+    gemm_ms = sum(prof[k][0] for k in ("gram", "poly", "update", "update_final"))
+    gemm_launches = sum(prof[k][1] for k in ("gram", "poly", "update", "update_final"))
+    row_kernel_ms = prof["row_wide"][0] + prof["row_tall"][0]
+    out = {
+        "metric": METRIC, "value": amort / world, "unit": "ms/step", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if args.check_mode else "bf16", "data": "synthetic",
+        "config": {"workload": wl.name, "K": K, "matrices": n, "blocks": wl.blocks, "d": wl.d,
+                   "elements": el, "io_dtype": wl.io_dtype, "momentum_dtype": "fp32",
+                   "ns5": "fp32 check mode" if args.check_mode else "bf16 tcgen05",
+                   "replicas": world, "l2": "inputs larger than L2 (working set %.1f GB)" % (el * 8 / 1e9),
+                   "first_timed_step_index": t_first + args.warmup},
+        "refresh_ms": mean_ref if n_ref else None, "row_step_ms": mean_row if n_row else None,
+        "refresh_steps_timed": n_ref, "row_steps_timed": n_row,
+        "gpu_launches": launches,
+        "clocks": clocks,
+    }
+    if n_row:
+        gbs = row_bytes / (mean_row * 1e-3) / 1e9
+        out["row_step"] = {"GB/s": gbs, "bytes_per_element": 3 * io_bytes + 8,
+                           "frac_of_measured_peak": gbs / pk["hbm_gbs"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+                           "kernel_ms_per_step": row_kernel_ms / n_row}
+    if n_ref and gemm_ms > 0:
+        tf_exec = ex * n_ref / (gemm_ms * 1e-3) / 1e12
+        out["ns5"] = {"TFLOP/s_exec": tf_exec, "TFLOP/s_model": mo * n_ref / (gemm_ms * 1e-3) / 1e12,
+                      "TFLOP/s_exec_whole_refresh": ex / (mean_ref * 1e-3) / 1e12,
+                      "frac_of_measured_burst": tf_exec / pk["bf16_tflops"],
+                      "frac_of_measured_sustained": tf_exec / pk["bf16_tflops_sustained"],
+                      "frac_of_nominal_2250": tf_exec / NOMINAL_BF16_TFLOPS,
+                      "gemm_ms_per_refresh": gemm_ms / n_ref, "prepass_ms_per_refresh": prof["prepass"][0] / n_ref}
+        if args.check_mode:
+            # fp32 FMA path: bounded by CUDA-core arithmetic, not by tensor cores
+            peak = 148 * 128 * 2 * 1.965e9 / 1e12
+            out["roofline"] = {"bound": "alu", "achieved": tf_exec, "peak": peak, "unit": "TFLOP/s",
+                               "frac": tf_exec / peak, "traffic": None, "kernel": "gemm_simt_kernel",
+                               "peak_source": "148 SMs x 128 fp32 FMA lanes x 2 flop x 1.965 GHz"}
+        else:
+            peak = pk["bf16_tflops_sustained"]
+            out["roofline"] = {"bound": "tensor", "achieved": tf_exec, "peak": peak, "unit": "TFLOP/s",
+                               "frac": tf_exec / peak, "traffic": None, "kernel": "gemm_tc_kernel",
+                               "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(1, gemm_launches),
+                               "peak_source": "%s sustained bf16 matmul" % pk["source"]}
+    elif n_row:
+        gbs = row_bytes / (row_kernel_ms / n_row * 1e-3) / 1e9
+        out["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                           "frac": gbs / pk["hbm_gbs"], "traffic": None, "kernel": "rowstep_*",
+                           "peak_source": "%s copy bandwidth" % pk["source"]}
+    out["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        out["cpu_baseline"] = oracle_sample(wl, K)
+    print(json.dumps(out))
+    if dist:
+        td.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

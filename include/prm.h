@@ -138,6 +138,25 @@ PRM_API const char* prm_last_error(const prm_ctx* ctx);
 /* Number of kernels the library has launched through this handle so far. */
 PRM_API int64_t prm_launch_count(const prm_ctx* ctx);
 
+/*
+ * Optional per-kernel-class device timing.  prm_profile(ctx, 1) makes every
+ * following prm_step bracket each kernel class with CUDA events on the step's
+ * stream (no device memory is allocated); prm_profile(ctx, 0) stops it.
+ * prm_profile_read waits for the recorded events and adds up, per class, the
+ * elapsed milliseconds and the number of kernel launches since the last read.
+ * ms and launches are host arrays of n_classes entries (PRM_PROF_COUNT).
+ */
+#define PRM_PROF_ROW_WIDE      0  /* fused row step, wide matrices */
+#define PRM_PROF_ROW_TALL      1  /* row step, tall matrices (3 kernels) */
+#define PRM_PROF_PREPASS       2  /* NS5 pre-pass and norm (2 kernels) */
+#define PRM_PROF_GRAM          3  /* A = X X^T */
+#define PRM_PROF_POLY          4  /* B = b A + c A^2 */
+#define PRM_PROF_UPDATE        5  /* X <- a X + B X */
+#define PRM_PROF_UPDATE_FINAL  6  /* last X update fused with the parameter update */
+#define PRM_PROF_COUNT         7
+PRM_API int prm_profile(prm_ctx* ctx, int enable);
+PRM_API int prm_profile_read(prm_ctx* ctx, double* ms, int64_t* launches, int n_classes);
+
 /* Frees host resources.  Device memory belongs to the caller. */
 PRM_API int prm_destroy(prm_ctx* ctx);
 

@@ -39,7 +39,11 @@ PRM_OPT_NS_WORKSPACE_BYTES = 9
 EXPORTS = (
     "prm_create", "prm_set_option", "prm_workspace_bytes", "prm_set_workspace", "prm_step",
     "prm_step_h2d", "prm_plan", "prm_status", "prm_last_error", "prm_launch_count", "prm_destroy",
+    "prm_profile", "prm_profile_read",
 )
+PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
+PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_COUNT = 4, 5, 6, 7
+PROF_NAMES = ("row_wide", "row_tall", "prepass", "gram", "poly", "update", "update_final")
 
 _lib_handle = None
 
@@ -83,6 +87,10 @@ def lib():
     L.prm_launch_count.restype = c_int64
     L.prm_destroy.argtypes = [c_void_p]
     L.prm_destroy.restype = c_int
+    L.prm_profile.argtypes = [c_void_p, c_int]
+    L.prm_profile.restype = c_int
+    L.prm_profile_read.argtypes = [c_void_p, POINTER(c_double), POINTER(c_int64), c_int]
+    L.prm_profile_read.restype = c_int
     _lib_handle = L
     return L
 
@@ -147,6 +155,17 @@ def prm_last_error(h):
 
 def prm_launch_count(h):
     return int(lib().prm_launch_count(h))
+
+
+def prm_profile(h, enable):
+    _check(lib().prm_profile(h, int(bool(enable))), h)
+
+
+def prm_profile_read(h):
+    ms = (c_double * PRM_PROF_COUNT)()
+    n = (c_int64 * PRM_PROF_COUNT)()
+    _check(lib().prm_profile_read(h, ms, n, PRM_PROF_COUNT), h)
+    return {name: (ms[i], n[i]) for i, name in enumerate(PROF_NAMES)}
 
 
 def prm_destroy(h):
@@ -222,6 +241,15 @@ class PeriodicRowwiseMuon:
 
     def status(self):
         return prm_status(self.h)
+
+    def profile(self, enable=True):
+        with torch.cuda.device(self.device):
+            prm_profile(self.h, enable)
+
+    def profile_read(self):
+        """{class name: (milliseconds, launches)} since the last read."""
+        with torch.cuda.device(self.device):
+            return prm_profile_read(self.h)
 
     def launch_count(self):
         return prm_launch_count(self.h)

@@ -37,7 +37,39 @@ struct prm_ctx {
   TcContext* tc = nullptr;
   std::string err;
   int64_t launches = 0;
+
+  // optional per-class device timing (prm_profile)
+  bool prof_on = false;
+  std::vector<cudaEvent_t> prof_ev;     // begin/end pairs
+  std::vector<int> prof_cls;            // class of pair i
+  std::vector<int64_t> prof_launches;   // kernel launches inside pair i
+  size_t prof_used = 0;
+  int64_t prof_dropped = 0;
 };
+
+namespace {
+constexpr size_t kProfPairs = 8192;
+
+struct ProfScope {
+  prm_ctx* c;
+  cudaStream_t stream;
+  long idx = -1;
+  int64_t launches0 = 0;
+  ProfScope(prm_ctx* ctx, int cls, cudaStream_t st) : c(ctx), stream(st) {
+    if (!c->prof_on) return;
+    if (c->prof_used >= kProfPairs) { c->prof_dropped++; return; }
+    idx = (long)c->prof_used++;
+    c->prof_cls[idx] = cls;
+    launches0 = c->launches;
+    cudaEventRecord(c->prof_ev[2 * idx], stream);
+  }
+  ~ProfScope() {
+    if (idx < 0) return;
+    cudaEventRecord(c->prof_ev[2 * idx + 1], stream);
+    c->prof_launches[idx] = c->launches - launches0;
+  }
+};
+}  // namespace
 
 static std::string g_create_err;
 
@@ -204,10 +236,15 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
     char* A = base + 4 * e * rc * nb;
     char* B = A + e * rr * nb;
     const int first = g.first + done;
-    cudaError_t ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, c->check_mode, X[0], XT[0],
-                                       fro, alpha, stream, &c->launches);
+    cudaError_t ce;
+    {
+      ProfScope ps(c, PRM_PROF_PREPASS, stream);
+      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, c->check_mode, X[0], XT[0], fro, alpha,
+                             stream, &c->launches);
+    }
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("pre-pass: ") + cudaGetErrorString(ce));
-    auto gemm = [&](const GemmProblem& pb, const Epilogue& ep) -> cudaError_t {
+    auto gemm = [&](const GemmProblem& pb, const Epilogue& ep, int cls) -> cudaError_t {
+      ProfScope ps(c, cls, stream);
       return c->check_mode ? launch_gemm_simt(pb, ep, stream, &c->launches)
                            : launch_gemm_tc(c->tc, pb, ep, status, stream, &c->launches);
     };
@@ -221,7 +258,7 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
       ea.dst = A; ea.ld_dst = g.rp; ea.bs_dst = rr;
       ea.dst_t = A; ea.ld_dst_t = g.rp; ea.bs_dst_t = rr;
       if (it == 0) { ea.alpha = alpha; ea.alpha_pow = 2; }
-      if ((ce = gemm(pa, ea)) != cudaSuccess) break;
+      if ((ce = gemm(pa, ea, PRM_PROF_GRAM)) != cudaSuccess) break;
       // B = b A + c A^2
       GemmProblem pp;
       pp.P = A; pp.Q = A; pp.Mp = g.rp; pp.Np = g.rp; pp.Kp = g.rp;
@@ -230,7 +267,7 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
       eb.k_acc = kNsC; eb.k_aux = kNsB; eb.aux = A; eb.ld_aux = g.rp; eb.bs_aux = rr;
       eb.dst = B; eb.ld_dst = g.rp; eb.bs_dst = rr;
       eb.dst_t = B; eb.ld_dst_t = g.rp; eb.bs_dst_t = rr;
-      if ((ce = gemm(pp, eb)) != cudaSuccess) break;
+      if ((ce = gemm(pp, eb, PRM_PROF_POLY)) != cudaSuccess) break;
       // X <- a X + B X (times alpha in the first iteration); last iteration
       // goes straight into the parameters.
       GemmProblem pu;
@@ -247,7 +284,7 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
         eu.rows = (int)g.rows; eu.cols = (int)g.cols; eu.tall = g.tall ? 1 : 0;
         eu.io_fp32 = c->io_fp32; eu.decay = s.decay; eu.lr_s = s.lr_s;
       }
-      if ((ce = gemm(pu, eu)) != cudaSuccess) break;
+      if ((ce = gemm(pu, eu, it + 1 < kNsIters ? PRM_PROF_UPDATE : PRM_PROF_UPDATE_FINAL)) != cudaSuccess) break;
       cur ^= 1;
     }
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("NS5 product: ") + cudaGetErrorString(ce));
@@ -307,6 +344,7 @@ static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
       int rc = refresh_group(c, g, t, s, stream);
       if (rc != PRM_OK) return rc;
     } else {
+      ProfScope ps(c, g.tall ? PRM_PROF_ROW_TALL : PRM_PROF_ROW_WIDE, stream);
       ce = launch_rowstep(t, g, s, c->io_fp32, (float*)(c->ws + g.tall_scratch_off),
                           (float*)(c->ws + g.tall_nu_off), stream, &c->launches);
       if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("row step: ") + cudaGetErrorString(ce));
@@ -339,6 +377,44 @@ extern "C" int prm_status(prm_ctx* c) {
   return PRM_OK;
 }
 
+extern "C" int prm_profile(prm_ctx* c, int enable) {
+  if (!c) return PRM_ERR_ARG;
+  if (enable && c->prof_ev.empty()) {
+    c->prof_ev.resize(2 * kProfPairs);
+    for (size_t i = 0; i < c->prof_ev.size(); ++i) {
+      cudaError_t ce = cudaEventCreate(&c->prof_ev[i]);
+      if (ce != cudaSuccess) {
+        for (size_t k = 0; k < i; ++k) cudaEventDestroy(c->prof_ev[k]);
+        c->prof_ev.clear();
+        return fail(c, PRM_ERR_CUDA, std::string("prm_profile: ") + cudaGetErrorString(ce));
+      }
+    }
+    c->prof_cls.assign(kProfPairs, 0);
+    c->prof_launches.assign(kProfPairs, 0);
+  }
+  c->prof_on = enable != 0;
+  c->prof_used = 0;
+  c->prof_dropped = 0;
+  return PRM_OK;
+}
+
+extern "C" int prm_profile_read(prm_ctx* c, double* ms, int64_t* launches, int n_classes) {
+  if (!c || !ms || !launches || n_classes < 1) return PRM_ERR_ARG;
+  for (int k = 0; k < n_classes; ++k) { ms[k] = 0.0; launches[k] = 0; }
+  for (size_t i = 0; i < c->prof_used; ++i) {
+    cudaError_t ce = cudaEventSynchronize(c->prof_ev[2 * i + 1]);
+    float t = 0.f;
+    if (ce == cudaSuccess) ce = cudaEventElapsedTime(&t, c->prof_ev[2 * i], c->prof_ev[2 * i + 1]);
+    if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("prm_profile_read: ") + cudaGetErrorString(ce));
+    const int cls = c->prof_cls[i];
+    if (cls < n_classes) { ms[cls] += t; launches[cls] += c->prof_launches[i]; }
+  }
+  const bool dropped = c->prof_dropped != 0;
+  c->prof_used = 0;
+  c->prof_dropped = 0;
+  return dropped ? fail(c, PRM_ERR_STATE, "prm_profile_read: event pool overflowed, totals incomplete") : PRM_OK;
+}
+
 extern "C" const char* prm_last_error(const prm_ctx* c) { return c ? c->err.c_str() : g_create_err.c_str(); }
 
 extern "C" int64_t prm_launch_count(const prm_ctx* c) { return c ? c->launches : 0; }
@@ -346,6 +422,7 @@ extern "C" int64_t prm_launch_count(const prm_ctx* c) { return c ? c->launches :
 extern "C" int prm_destroy(prm_ctx* c) {
   if (!c) return PRM_ERR_ARG;
   if (c->tc) tc_destroy(c->tc);
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
   delete c;
   return PRM_OK;
 }

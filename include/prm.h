@@ -157,6 +157,44 @@ PRM_API int64_t prm_launch_count(const prm_ctx* ctx);
 PRM_API int prm_profile(prm_ctx* ctx, int enable);
 PRM_API int prm_profile_read(prm_ctx* ctx, double* ms, int64_t* launches, int n_classes);
 
+/*
+ * Row step of ONE tall matrix (rows > cols) that allocates nothing.  (The
+ * paper has no counterpart: this entry point exists for the library's users,
+ * not for the method.)
+ *
+ * It is meant for callers that cannot allocate device memory and so cannot
+ * give prm_step a workspace: code running inside a process whose memory pool
+ * already owns the GPU's memory, or a loop that must stay clear of the
+ * device-wide synchronisation inside cudaMalloc/cudaFree.  The column
+ * partial sums and column norms that the tall row step needs live in a fixed
+ * 4 MiB array inside the library image (held by every GPU that loads the
+ * library, until the process exits).  The call itself performs no cudaMalloc,
+ * cudaFree or other allocating call.
+ *
+ *   param, grad   device pointers, rows x cols row-major, bf16 (io_fp32 = 0)
+ *                 or fp32 (io_fp32 = 1); param is updated in place
+ *   momentum      device pointer, fp32, updated in place
+ *   scale         the shape factor s(W) to apply (e.g. sqrt(rows/cols))
+ *   other scalars as in prm_create / prm_set_option
+ *   errbuf        optional host buffer for an error text (may be NULL)
+ * Computes exactly what prm_step computes for a tall matrix on a non-refresh
+ * step.  Limits: cols a multiple of 8, and (ceil(rows/128) + 1) * cols <=
+ * 1048576 floats; larger matrices are refused with PRM_ERR_WORKSPACE and a
+ * message, before anything is launched.  Wide matrices are refused with
+ * PRM_ERR_SHAPE (their row step needs no scratch).
+ *
+ * The first call on each device looks up the array's device address (with that
+ * device current); make that first call outside any stream capture.  All
+ * calls share the one array: it keeps the previous call's contents, none of
+ * which is read before being overwritten, and calls that overlap on the GPU
+ * (different streams without ordering) race on it.
+ */
+PRM_API int prm_rowstep_tall_noalloc(void* param, const void* grad, float* momentum,
+                                     int64_t rows, int64_t cols, int io_fp32, float beta,
+                                     int nesterov, float lr, float wd, float gamma, float eps_row,
+                                     float scale, void* cuda_stream, char* errbuf,
+                                     size_t errbuf_len);
+
 /* Frees host resources.  Device memory belongs to the caller. */
 PRM_API int prm_destroy(prm_ctx* ctx);
 

@@ -39,7 +39,7 @@ PRM_OPT_NS_WORKSPACE_BYTES = 9
 EXPORTS = (
     "prm_create", "prm_set_option", "prm_workspace_bytes", "prm_set_workspace", "prm_step",
     "prm_step_h2d", "prm_plan", "prm_status", "prm_last_error", "prm_launch_count", "prm_destroy",
-    "prm_profile", "prm_profile_read",
+    "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc",
 )
 PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
 PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_COUNT = 4, 5, 6, 7
@@ -91,6 +91,10 @@ def lib():
     L.prm_profile.restype = c_int
     L.prm_profile_read.argtypes = [c_void_p, POINTER(c_double), POINTER(c_int64), c_int]
     L.prm_profile_read.restype = c_int
+    L.prm_rowstep_tall_noalloc.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int, c_float,
+                                           c_int, c_float, c_float, c_float, c_float, c_float, c_void_p,
+                                           c_char_p, c_size_t]
+    L.prm_rowstep_tall_noalloc.restype = c_int
     _lib_handle = L
     return L
 
@@ -166,6 +170,25 @@ def prm_profile_read(h):
     n = (c_int64 * PRM_PROF_COUNT)()
     _check(lib().prm_profile_read(h, ms, n, PRM_PROF_COUNT), h)
     return {name: (ms[i], n[i]) for i, name in enumerate(PROF_NAMES)}
+
+
+def prm_rowstep_tall_noalloc(param, grad, momentum, *, beta, nesterov, lr, wd, gamma, eps_row, scale,
+                             stream=None):
+    """Row step of one tall matrix for callers that cannot allocate device
+    memory (no workspace, no handle): the scratch sits in a fixed array inside
+    the library.  Tensors are updated in place; see include/prm.h for the size
+    limit and the sharing rules of that array."""
+    rows, cols = param.shape
+    io_fp32 = 1 if param.dtype == torch.float32 else 0
+    s = (stream or torch.cuda.current_stream(param.device)).cuda_stream
+    buf = ctypes.create_string_buffer(256)
+    with torch.cuda.device(param.device):
+        code = lib().prm_rowstep_tall_noalloc(
+            c_void_p(param.data_ptr()), c_void_p(grad.data_ptr()), c_void_p(momentum.data_ptr()),
+            int(rows), int(cols), io_fp32, float(beta), int(bool(nesterov)), float(lr), float(wd),
+            float(gamma), float(eps_row), float(scale), c_void_p(s), buf, 256)
+    if code != PRM_OK:
+        raise PrmError(code, buf.value.decode())
 
 
 def prm_destroy(h):

@@ -1,0 +1,72 @@
+"""The allocation-free row step for tall matrices against the regular path.
+
+Some users of this library cannot allocate device memory at all (their host
+process has already handed the whole GPU to its own memory pool, or they run
+in a loop that must not take the device-wide stall of cudaMalloc), so they
+cannot attach the workspace that `prm_step` needs for the column norms of
+tall matrices.  `prm_rowstep_tall_noalloc` serves them from a fixed array
+inside the library.  This file checks that it computes what `prm_step`
+computes, on two calls in a row that share that array, and that it refuses
+matrices too large for it.  It is collected last on purpose.
+"""
+
+import math
+
+import pytest
+import torch
+
+from paper_2608_20818_b200 import binding as B
+from tests import util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _both_paths(shape, io, nesterov, seed):
+    cfg = U.oracle_cfg(K=4, beta=0.95, nesterov=nesterov, lr=5e-3, wd=0.01, gamma=0.15, eps_row=1e-8)
+    W, G, M = U.make_inputs([shape], seed, io)
+    # existing entry point (workspace allocated by torch)
+    W_ref, M_ref = U.gpu_step([shape], W, G, M, t=1, cfg=cfg, io=io, check_mode=True)
+    # new entry point: no workspace, no handle
+    w, g, m = U.Guarded(W[0]), U.Guarded(G[0]), U.Guarded(M[0])
+    before = torch.cuda.memory_allocated()
+    B.prm_rowstep_tall_noalloc(w.t, g.t, m.t, beta=cfg.beta, nesterov=cfg.nesterov, lr=cfg.lr, wd=cfg.wd,
+                               gamma=cfg.gamma, eps_row=cfg.eps_row,
+                               scale=math.sqrt(max(1.0, shape[0] / shape[1])))
+    torch.cuda.synchronize()
+    assert torch.cuda.memory_allocated() == before
+    assert w.intact() and g.intact() and m.intact()
+    assert torch.equal(g.t.cpu(), G[0])
+    U.assert_elementwise(U.to_np64(m.t), M_ref[0], False, f"momentum {shape}")
+    U.assert_elementwise(U.to_np64(w.t), W_ref[0], io == "bf16", f"param {shape}")
+
+
+def test_no_alloc_matches_step_on_two_calls_in_a_row():
+    # the second call is smaller and of the other storage type, so it runs on
+    # an array that still holds the first call's partial sums
+    _both_paths((2048, 512), "bf16", True, seed=21)
+    _both_paths((1000, 264), "fp32", False, seed=22)
+    _both_paths((2048, 512), "bf16", True, seed=23)
+
+
+def test_no_alloc_refuses_what_does_not_fit():
+    big = (300000, 512)          # (ceil(rows/128)+1)*cols = 1.2M floats > 1M
+    p = torch.zeros(8, 8, dtype=torch.bfloat16, device="cuda")
+    m = torch.zeros(8, 8, device="cuda")
+
+    class Fake:
+        def __init__(self, t, shape):
+            self.t, self.shape, self.dtype, self.device = t, shape, t.dtype, t.device
+
+        def data_ptr(self):
+            return self.t.data_ptr()
+
+    with pytest.raises(B.PrmError) as e:
+        B.prm_rowstep_tall_noalloc(Fake(p, big), Fake(p, big), Fake(m, big), beta=0.95, nesterov=True,
+                                   lr=1e-3, wd=0.0, gamma=0.15, eps_row=1e-8, scale=1.0)
+    assert e.value.code == B.PRM_ERR_WORKSPACE and "scratch" in str(e.value)
+    with pytest.raises(B.PrmError) as e:
+        B.prm_rowstep_tall_noalloc(Fake(p, (8, 8)), Fake(p, (8, 8)), Fake(m, (8, 8)), beta=0.95, nesterov=True,
+                                   lr=1e-3, wd=0.0, gamma=0.15, eps_row=1e-8, scale=1.0)
+    assert e.value.code == B.PRM_ERR_SHAPE
+    torch.cuda.synchronize()
+    assert not p.any() and not m.any()

@@ -1,15 +1,366 @@
-// Tensor-core NS5 products (placeholder until the tcgen05 kernel lands).
+// Tensor-core NS5 products for sm_100a: D[i,j] = sum_k P[i,k]*Q[j,k] with bf16
+// operands, fp32 accumulation in tensor memory, and the fused epilogues of
+// struct Epilogue (polynomial coefficients, Frobenius scale, mirror write,
+// transposed copy of X, final parameter update).
+//
+// One persistent CTA per SM, 192 threads:
+//   warp 0      TMA producer: 128x64 tile of P and 256x64 tile of Q per stage
+//               (cp.async.bulk.tensor, 128-byte swizzle, no multicast)
+//   warp 1      tcgen05.mma issuer (one lane), owns the TMEM allocation
+//   warps 2..5  epilogue: tcgen05.ld of a 128x256 fp32 accumulator, fused
+//               arithmetic, global stores
+// Two 256-column accumulators in TMEM let the epilogue of tile n overlap the
+// main loop of tile n+1.  Every mbarrier wait is bounded: on expiry the CTA
+// raises the status word, drains and exits cleanly.
+#include <cuda.h>
+
+#include <map>
+#include <tuple>
+
 #include "epilogue.cuh"
 
 namespace prm {
 
-struct TcContext { int unused; };
+namespace {
 
-TcContext* tc_create(std::string* err) { (void)err; return new TcContext(); }
+constexpr int kBM = 128;          // tile rows  (UMMA M)
+constexpr int kBN = 256;          // tile cols  (UMMA N)
+constexpr int kBK = 64;           // k per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaK = 16;
+constexpr int kStages = 4;
+constexpr int kTcThreads = 192;
+constexpr uint32_t kBytesA = kBM * kBK * 2;
+constexpr uint32_t kBytesB = kBN * kBK * 2;
+constexpr uint32_t kStageBytes = kBytesA + kBytesB;
+constexpr uint32_t kTmemCols = 512;
+constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) |
+                            ((uint32_t)(kBM >> 4) << 24);
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting (this or another role
+// ran out of time); the first to give up raises the device status word.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      atomicOr(status, kStatusTimeout);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int x,
+                                            int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
+  // K-major operand tile, 128-byte swizzle: rows of 128 bytes, groups of 8
+  // rows 1024 bytes apart (stride byte offset), descriptor version 1.
+  return (uint64_t)((smem_addr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+struct TileCoord {
+  int b, ti, tj;
+  bool mirror;
+};
+__device__ __forceinline__ TileCoord decode_tile(int t, int tiles_per_mat, int symmetric, int mt) {
+  TileCoord c;
+  c.b = t / tiles_per_mat;
+  const int rem = t - c.b * tiles_per_mat;
+  if (symmetric) {
+    int bi, bj;
+    tri_decode(rem >> 1, bi, bj);      // 256x256 blocks of the lower triangle
+    c.ti = 2 * bi + (rem & 1);         // two 128-row tiles per block
+    c.tj = bj;
+    c.mirror = bi != bj;
+  } else {
+    c.ti = rem % mt;                   // row tiles fastest: concurrent CTAs share the Q panel
+    c.tj = rem / mt;
+    c.mirror = true;
+  }
+  return c;
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ,
+               int ktiles, int tiles_per_mat, int total_tiles, int symmetric, int mt, Epilogue ep,
+               int* status) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes);
+  uint64_t* full = bars;                      // [kStages] TMA -> MMA
+  uint64_t* empty = bars + kStages;           // [kStages] MMA -> TMA
+  uint64_t* tfull = bars + 2 * kStages;       // [2] MMA -> epilogue
+  uint64_t* tempty = bars + 2 * kStages + 2;  // [2] epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 4); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ producer
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
+        const TileCoord c = decode_tile(t, tiles_per_mat, symmetric, mt);
+        for (int kt = 0; kt < ktiles; ++kt, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1;
+          if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, status)) { ok = false; break; }
+          uint8_t* sa = smem + (size_t)s * kStageBytes;
+          mbar_expect_tx(&full[s], kStageBytes);
+          tma_load_3d(sa, &mapP, &full[s], kt * kBK, c.ti * kBM, c.b);
+          tma_load_3d(sa + kBytesA, &mapQ, &full[s], kt * kBK, c.tj * kBN, c.b);
+        }
+      }
+      // Drain: every load issued must have landed before shared memory is released.
+      const uint32_t n_issued = it;
+      for (uint32_t k = (n_issued > kStages ? n_issued - kStages : 0); k < n_issued; ++k) {
+        const uint64_t t0 = global_ns();
+        while (!mbar_try_wait(&full[k % kStages], (k / kStages) & 1)) {
+          if (global_ns() - t0 > 1000000ull) break;   // 1 ms
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // -------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, acc_it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_it) {
+        const int a = acc_it & 1;
+        const uint32_t aph = (acc_it >> 1) & 1;
+        if (!mbar_wait(&tempty[a], aph ^ 1, abort_flag, status)) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t tacc = tmem_base + (uint32_t)a * kBN;
+        for (int kt = 0; kt < ktiles; ++kt, ++it) {
+          const int s = it % kStages;
+          const uint32_t ph = (it / kStages) & 1;
+          if (!mbar_wait(&full[s], ph, abort_flag, status)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
+          const uint64_t da = make_desc(sa), db = make_desc(sa + kBytesA);
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            // advance 16 elements = 32 bytes inside the swizzled row: +2 in 16-byte units
+            umma_bf16(tacc, da + 2 * k, db + 2 * k, (kt | k) != 0);
+          }
+          umma_commit(&empty[s]);        // frees the stage when these MMAs have read it
+        }
+        if (ok) umma_commit(&tfull[a]);  // accumulator complete
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- epilogue
+    const int q = warp & 3;              // TMEM lane quadrant this warp may read
+    uint32_t acc_it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_it) {
+      const TileCoord c = decode_tile(t, tiles_per_mat, symmetric, mt);
+      const int a = acc_it & 1;
+      const uint32_t aph = (acc_it >> 1) & 1;
+      // All lanes wait, then agree: tcgen05.ld needs the whole warp.
+      const bool got = mbar_wait(&tfull[a], aph, abort_flag, status);
+      if (!__all_sync(0xffffffffu, got)) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int i = c.ti * kBM + q * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)a * kBN;
+#pragma unroll 1
+      for (int ch = 0; ch < kBN / 32; ++ch) {
+        float v[32];
+        tmem_ld32(taddr + ch * 32, v);
+        epilogue_row<__nv_bfloat16, 32>(ep, c.b, i, c.tj * kBN + ch * 32, v, c.mirror);
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[a]);
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct TcContext {
+  EncodeTiledFn encode = nullptr;
+  int sm_count = 0;
+  std::map<std::tuple<const void*, int64_t, int64_t, int, int>, CUtensorMap> cache;
+};
+
+TcContext* tc_create(std::string* err) {
+  TcContext* tc = new TcContext();
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t ce = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (ce != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+    if (err) *err = "cuTensorMapEncodeTiled is not available from the driver";
+    delete tc;
+    return nullptr;
+  }
+  tc->encode = (EncodeTiledFn)fn;
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    if (err) *err = "cannot query the CUDA device";
+    delete tc;
+    return nullptr;
+  }
+  if (prop.major != 10) {
+    if (err) *err = "the tensor-core path needs an sm_100 device";
+    delete tc;
+    return nullptr;
+  }
+  tc->sm_count = prop.multiProcessorCount;
+  ce = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (ce != cudaSuccess) {
+    if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(ce);
+    delete tc;
+    return nullptr;
+  }
+  return tc;
+}
+
 void tc_destroy(TcContext* tc) { delete tc; }
 
-cudaError_t launch_gemm_tc(TcContext*, const GemmProblem&, const Epilogue&, int*, cudaStream_t, int64_t*) {
-  return cudaErrorNotSupported;
+// 3-D map over a [batch][rows][kdim] bf16 array; box = 64 (k) x box_rows x 1.
+static bool get_map(TcContext* tc, const void* base, int64_t rows, int64_t kdim, int batch, int box_rows,
+                    CUtensorMap* out) {
+  auto key = std::make_tuple(base, rows, kdim, batch, box_rows);
+  auto it = tc->cache.find(key);
+  if (it != tc->cache.end()) { *out = it->second; return true; }
+  cuuint64_t dims[3] = {(cuuint64_t)kdim, (cuuint64_t)rows, (cuuint64_t)batch};
+  cuuint64_t strides[2] = {(cuuint64_t)kdim * 2, (cuuint64_t)kdim * (cuuint64_t)rows * 2};
+  cuuint32_t box[3] = {(cuuint32_t)kBK, (cuuint32_t)box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = tc->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (tc->cache.size() > 4096) tc->cache.clear();
+  tc->cache[key] = *out;
+  return true;
+}
+
+cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue& ep, int* status,
+                           cudaStream_t stream, int64_t* launches) {
+  if (!tc) return cudaErrorInvalidValue;
+  if (pb.Mp % kBN != 0 || pb.Np % kBN != 0 || pb.Kp % kBK != 0) return cudaErrorInvalidValue;
+  CUtensorMap mp, mq;
+  if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
+  if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN, &mq)) return cudaErrorInvalidValue;
+  const int64_t mt = pb.Mp / kBM, nt = pb.Np / kBN;
+  int64_t per_mat;
+  if (pb.symmetric) {
+    const int64_t nb = pb.Mp / kBN;          // 256x256 blocks per side
+    per_mat = nb * (nb + 1);                 // lower-triangle blocks x 2 row tiles
+  } else {
+    per_mat = mt * nt;
+  }
+  const int64_t total = per_mat * pb.batch;
+  if (total > 0x7fffffffLL) return cudaErrorInvalidValue;
+  const int grid = (int)std::min<int64_t>(total, tc->sm_count);
+  *launches += 1;
+  gemm_tc_kernel<<<grid, kTcThreads, kSmemBytes, stream>>>(mp, mq, (int)(pb.Kp / kBK), (int)per_mat, (int)total,
+                                                           pb.symmetric, (int)mt, ep, status);
+  return cudaGetLastError();
 }
 
 }  // namespace prm

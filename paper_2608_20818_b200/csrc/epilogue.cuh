@@ -7,9 +7,11 @@
 namespace prm {
 
 // XT_: element type of the workspace arrays (bf16 or float).  N multiple of 8.
+// pre: optional N auxiliary values already fetched by the caller (see
+// aux_prefetch); when null the auxiliary operand is loaded here.
 template <typename XT_, int N>
 __device__ __forceinline__ void epilogue_row(const Epilogue& ep, int b, int i, int j0,
-                                             float (&acc)[N], bool mirror) {
+                                             float (&acc)[N], bool mirror, const float* pre = nullptr) {
   const float al = ep.alpha ? ep.alpha[b] : 1.f;
   const float f = ep.alpha_pow == 2 ? al * al : (ep.alpha_pow == 1 ? al : 1.f);
   const float ka = f * ep.k_acc, kx = f * ep.k_aux;
@@ -19,7 +21,12 @@ __device__ __forceinline__ void epilogue_row(const Epilogue& ep, int b, int i, i
 #pragma unroll
     for (int v = 0; v < N; v += 8) {
       float x[8];
-      load8(aux + v, x);
+      if (pre != nullptr) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) x[e] = pre[v + e];
+      } else {
+        load8(aux + v, x);
+      }
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[v + e] = ka * acc[v + e] + kx * x[e];
     }
@@ -94,6 +101,33 @@ __device__ __forceinline__ void epilogue_row(const Epilogue& ep, int b, int i, i
           }
         }
       }
+    }
+  }
+}
+
+// N bf16 auxiliary values of one output row, fetched ahead of use.
+template <int N>
+struct AuxRegs {
+  int4 r[N / 8];
+};
+template <int N>
+__device__ __forceinline__ void aux_prefetch(const Epilogue& ep, int b, int i, int j0, AuxRegs<N>& a) {
+  if (ep.aux == nullptr) return;
+  const int4* p = reinterpret_cast<const int4*>(reinterpret_cast<const __nv_bfloat16*>(ep.aux) +
+                                                (int64_t)b * ep.bs_aux + (int64_t)i * ep.ld_aux + j0);
+#pragma unroll
+  for (int v = 0; v < N / 8; ++v) a.r[v] = p[v];
+}
+template <int N>
+__device__ __forceinline__ void aux_unpack(const AuxRegs<N>& a, float (&x)[N]) {
+#pragma unroll
+  for (int v = 0; v < N / 8; ++v) {
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&a.r[v]);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float2 f = __bfloat1622float2(h[k]);
+      x[8 * v + 2 * k] = f.x;
+      x[8 * v + 2 * k + 1] = f.y;
     }
   }
 }

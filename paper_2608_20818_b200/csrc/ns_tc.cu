@@ -3,15 +3,22 @@
 // struct Epilogue (polynomial coefficients, Frobenius scale, mirror write,
 // transposed copy of X, final parameter update).
 //
-// One persistent CTA per SM, 192 threads:
+// One persistent CTA per SM, 352 threads:
 //   warp 0      TMA producer: 128x64 tile of P and 256x64 tile of Q per stage
 //               (cp.async.bulk.tensor, 128-byte swizzle, no multicast)
 //   warp 1      tcgen05.mma issuer (one lane), owns the TMEM allocation
-//   warps 2..5  epilogue: tcgen05.ld of a 128x256 fp32 accumulator, fused
-//               arithmetic, global stores
-// Two 256-column accumulators in TMEM let the epilogue of tile n overlap the
-// main loop of tile n+1.  Every mbarrier wait is bounded: on expiry the CTA
-// raises the status word, drains and exits cleanly.
+//   warps 2..9  epilogue arithmetic: two warps per TMEM lane quadrant; the
+//               tile is finished in four slabs of 64 columns.  Per slab:
+//               tcgen05.ld of the fp32 accumulator, auxiliary operand read
+//               from a shared-memory slab, result written back in place and,
+//               transposed, into a second slab
+//   warp 10     epilogue I/O: TMA load of the auxiliary slab, TMA stores of
+//               the result slab and of its transpose
+// All global traffic of the product epilogues therefore moves as 128-byte
+// swizzled TMA boxes; per-thread global accesses remain only in the final
+// parameter update.  Two 256-column accumulators in TMEM let the epilogue of
+// tile n overlap the main loop of tile n+1.  Every mbarrier wait is bounded:
+// on expiry the CTA raises the status word, drains and exits cleanly.
 #include <cuda.h>
 
 #include <map>
@@ -27,14 +34,21 @@ constexpr int kBM = 128;          // tile rows  (UMMA M)
 constexpr int kBN = 256;          // tile cols  (UMMA N)
 constexpr int kBK = 64;           // k per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
-constexpr int kStages = 4;
-constexpr int kTcThreads = 192;
+constexpr int kStages = 3;
+constexpr int kEpiWarps = 8;         // two warps per TMEM lane quadrant
+constexpr int kIoWarp = 2 + kEpiWarps;
+constexpr int kTcThreads = 32 * (kIoWarp + 1);
+constexpr int kSlabCols = 64;        // epilogue slab: 128 rows x 64 columns
+constexpr int kSlabs = 4;            // slabs per tile (kBN / kSlabCols)
+constexpr int kEpiBufs = 2;
+constexpr uint32_t kSlabBytes = 128 * kSlabCols * 2;        // result slab, also the aux slab
+constexpr uint32_t kEpiBufBytes = 2 * kSlabBytes;           // + transposed slab (2 boxes of 64x64)
 constexpr uint32_t kBytesA = kBM * kBK * 2;
 constexpr uint32_t kBytesB = kBN * kBK * 2;
 constexpr uint32_t kStageBytes = kBytesA + kBytesB;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
-constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + (size_t)kEpiBufs * kEpiBufBytes + 256;
 
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128.
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) |
@@ -92,6 +106,18 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const void* src, const CUtensorMap* map, int x, int y, int z) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"((uint64_t)map), "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Byte offset of 16-byte chunk `chunk` of row `row` in a 128-byte-swizzled box.
+__device__ __forceinline__ uint32_t sw128(uint32_t row, uint32_t chunk) {
+  return row * 128u + ((chunk ^ (row & 7u)) << 4);
+}
 __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
   // K-major operand tile, 128-byte swizzle: rows of 128 bytes, groups of 8
   // rows 1024 bytes apart (stride byte offset), descriptor version 1.
@@ -110,8 +136,8 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                : "memory");
 }
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
-  uint32_t r[32];
+// Issues the TMEM load; the registers are valid after tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -121,9 +147,9 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
         "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
         "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 struct TileCoord {
@@ -150,23 +176,30 @@ __device__ __forceinline__ TileCoord decode_tile(int t, int tiles_per_mat, int s
 
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ,
-               int ktiles, int tiles_per_mat, int total_tiles, int symmetric, int mt, Epilogue ep,
-               int* status) {
+               const __grid_constant__ CUtensorMap mapAux, const __grid_constant__ CUtensorMap mapDst,
+               const __grid_constant__ CUtensorMap mapDstT, int ktiles, int tiles_per_mat,
+               int total_tiles, int symmetric, int mt, Epilogue ep, int* status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStages * kStageBytes);
+  uint8_t* ebuf = smem + (size_t)kStages * kStageBytes;           // [kEpiBufs][kEpiBufBytes]
+  uint64_t* bars = reinterpret_cast<uint64_t*>(ebuf + (size_t)kEpiBufs * kEpiBufBytes);
   uint64_t* full = bars;                      // [kStages] TMA -> MMA
-  uint64_t* empty = bars + kStages;           // [kStages] MMA -> TMA
-  uint64_t* tfull = bars + 2 * kStages;       // [2] MMA -> epilogue
-  uint64_t* tempty = bars + 2 * kStages + 2;  // [2] epilogue -> MMA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
+  uint64_t* empty = full + kStages;           // [kStages] MMA -> TMA
+  uint64_t* tfull = empty + kStages;          // [2] MMA -> epilogue
+  uint64_t* tempty = tfull + 2;               // [2] epilogue -> MMA
+  uint64_t* eready = tempty + 2;              // [kEpiBufs] I/O warp -> epilogue: slab buffer usable (aux landed)
+  uint64_t* edone = eready + kEpiBufs;        // [kEpiBufs] epilogue -> I/O warp: slab written
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(edone + kEpiBufs);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const bool staged = ep.kind == 0;           // product epilogue through shared memory and TMA
+  const bool has_aux = ep.aux != nullptr;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 4); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], kEpiWarps); }
+    for (int e = 0; e < kEpiBufs; ++e) { mbar_init(&eready[e], 1); mbar_init(&edone[e], kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -236,10 +269,61 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
         if (ok) umma_commit(&tfull[a]);  // accumulator complete
       }
     }
+  } else if (warp == kIoWarp) {
+    // ------------------------------------------------------------ epilogue I/O
+    // Slab g of this CTA (four per tile) lives in buffer g % kEpiBufs.  For
+    // each slab: make the buffer usable (load the auxiliary slab, or just
+    // signal), later store what the epilogue warps wrote.
+    if (lane == 0 && staged) {
+      int n_my_tiles = 0;
+      for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) ++n_my_tiles;
+      const uint32_t n_slabs = (uint32_t)n_my_tiles * kSlabs;
+      auto prepare = [&](uint32_t g) {
+        const int bsel = g % kEpiBufs;
+        if (has_aux) {
+          const TileCoord c = decode_tile(blockIdx.x + (int)(g / kSlabs) * gridDim.x, tiles_per_mat, symmetric, mt);
+          mbar_expect_tx(&eready[bsel], kSlabBytes);
+          tma_load_3d(ebuf + (size_t)bsel * kEpiBufBytes, &mapAux, &eready[bsel],
+                      c.tj * kBN + (int)(g % kSlabs) * kSlabCols, c.ti * kBM, c.b);
+        } else {
+          mbar_arrive(&eready[bsel]);
+        }
+      };
+      for (uint32_t g = 0; g < (uint32_t)kEpiBufs && g < n_slabs; ++g) prepare(g);
+      for (uint32_t g = 0; g < n_slabs; ++g) {
+        const int bsel = g % kEpiBufs;
+        if (!mbar_wait(&edone[bsel], (g / kEpiBufs) & 1, abort_flag, status)) break;
+        const TileCoord c = decode_tile(blockIdx.x + (int)(g / kSlabs) * gridDim.x, tiles_per_mat, symmetric, mt);
+        const int j0 = c.tj * kBN + (int)(g % kSlabs) * kSlabCols;
+        const uint8_t* buf = ebuf + (size_t)bsel * kEpiBufBytes;
+        tma_store_3d(buf, &mapDst, j0, c.ti * kBM, c.b);
+        if (c.mirror && ep.dst_t != nullptr) {
+          tma_store_3d(buf + kSlabBytes, &mapDstT, c.ti * kBM, j0, c.b);
+          tma_store_3d(buf + kSlabBytes + kSlabBytes / 2, &mapDstT, c.ti * kBM + 64, j0, c.b);
+        }
+        tma_store_commit();
+        if (g + kEpiBufs < n_slabs) {
+          tma_store_wait_read();          // the buffer has been read out: it can be refilled
+          prepare(g + kEpiBufs);
+        }
+      }
+      tma_store_wait_all();
+      if (has_aux) {
+        // Drain auxiliary loads that were issued but never consumed (abort path only).
+        for (int e = 0; e < kEpiBufs; ++e) {
+          const uint64_t t0 = global_ns();
+          while (*abort_flag && !mbar_try_wait(&eready[e], 0) && !mbar_try_wait(&eready[e], 1)) {
+            if (global_ns() - t0 > 1000000ull) break;
+          }
+        }
+      }
+    }
   } else {
     // ---------------------------------------------------------------- epilogue
     const int q = warp & 3;              // TMEM lane quadrant this warp may read
-    uint32_t acc_it = 0;
+    const int half = (warp - 2) >> 2;    // which half of the columns (of the slab, or of the tile)
+    const int row = q * 32 + lane;       // row of the tile owned by this thread
+    uint32_t acc_it = 0, g = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_it) {
       const TileCoord c = decode_tile(t, tiles_per_mat, symmetric, mt);
@@ -249,13 +333,81 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
       const bool got = mbar_wait(&tfull[a], aph, abort_flag, status);
       if (!__all_sync(0xffffffffu, got)) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const int i = c.ti * kBM + q * 32 + lane;
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)a * kBN;
+      const int i = c.ti * kBM + row;
+      const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * kBN);
+      if (staged) {
+        const float al = ep.alpha ? ep.alpha[c.b] : 1.f;
+        const float f = ep.alpha_pow == 2 ? al * al : (ep.alpha_pow == 1 ? al : 1.f);
+        const float ka = f * ep.k_acc, kx = f * ep.k_aux;
+        const bool write_t = c.mirror && ep.dst_t != nullptr;
 #pragma unroll 1
-      for (int ch = 0; ch < kBN / 32; ++ch) {
-        float v[32];
-        tmem_ld32(taddr + ch * 32, v);
-        epilogue_row<__nv_bfloat16, 32>(ep, c.b, i, c.tj * kBN + ch * 32, v, c.mirror);
+        for (int sl = 0; sl < kSlabs; ++sl, ++g) {
+          const int bsel = g % kEpiBufs;
+          uint32_t r[32];
+          tmem_ld32_issue(trow + sl * kSlabCols + half * 32, r);
+          const bool rdy = mbar_wait(&eready[bsel], (g / kEpiBufs) & 1, abort_flag, status);
+          tmem_ld_wait();
+          if (!__all_sync(0xffffffffu, rdy)) { ok = false; break; }
+          uint8_t* buf = ebuf + (size_t)bsel * kEpiBufBytes;
+          uint8_t* tbuf = buf + kSlabBytes + (row >> 6) * (kSlabBytes / 2);
+          const uint32_t rt = row & 63;
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            int4* p = reinterpret_cast<int4*>(buf + sw128(row, half * 4 + v));
+            float x[8];
+            if (has_aux) {
+              const int4 raw = *p;
+              const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float2 ff = __bfloat1622float2(h2[k]);
+                x[2 * k] = ff.x;
+                x[2 * k + 1] = ff.y;
+              }
+            } else {
+#pragma unroll
+              for (int k = 0; k < 8; ++k) x[k] = 0.f;
+            }
+            int4 outv;
+            __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&outv);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float v0 = ka * __uint_as_float(r[8 * v + 2 * k]) + kx * x[2 * k];
+              const float v1 = ka * __uint_as_float(r[8 * v + 2 * k + 1]) + kx * x[2 * k + 1];
+              o2[k] = __floats2bfloat162_rn(v0, v1);
+            }
+            *p = outv;
+            if (write_t) {
+              const __nv_bfloat16* o1 = reinterpret_cast<const __nv_bfloat16*>(&outv);
+#pragma unroll
+              for (int k = 0; k < 8; ++k) {
+                const uint32_t cc = half * 32 + v * 8 + k;     // column inside the slab = row of the transpose
+                *reinterpret_cast<__nv_bfloat16*>(tbuf + sw128(cc, rt >> 3) + (rt & 7) * 2) = o1[k];
+              }
+            }
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&edone[bsel]);
+        }
+      } else {
+        // Final parameter update: per-thread global accesses.
+        const int jbase = c.tj * kBN + half * (kBN / 2);
+        constexpr int kChunks = kBN / 2 / 32;
+        AuxRegs<32> aux[2];
+        aux_prefetch<32>(ep, c.b, i, jbase, aux[0]);
+#pragma unroll
+        for (int ch = 0; ch < kChunks; ++ch) {
+          uint32_t r[32];
+          tmem_ld32_issue(trow + half * (kBN / 2) + ch * 32, r);
+          if (ch + 1 < kChunks) aux_prefetch<32>(ep, c.b, i, jbase + (ch + 1) * 32, aux[(ch + 1) & 1]);
+          tmem_ld_wait();
+          float v[32], x[32];
+#pragma unroll
+          for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
+          aux_unpack<32>(aux[ch & 1], x);
+          epilogue_row<__nv_bfloat16, 32>(ep, c.b, i, jbase + ch * 32, v, c.mirror, x);
+        }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -343,9 +495,24 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
                            cudaStream_t stream, int64_t* launches) {
   if (!tc) return cudaErrorInvalidValue;
   if (pb.Mp % kBN != 0 || pb.Np % kBN != 0 || pb.Kp % kBK != 0) return cudaErrorInvalidValue;
-  CUtensorMap mp, mq;
+  CUtensorMap mp, mq, maux, mdst, mdt;
   if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
   if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN, &mq)) return cudaErrorInvalidValue;
+  // Epilogue maps (product epilogues only): auxiliary and result slabs of 128
+  // rows x 64 columns, transposed result in boxes of 64 x 64.
+  maux = mp; mdst = mp; mdt = mp;
+  if (ep.kind == 0) {
+    if (ep.bs_dst != pb.Mp * ep.ld_dst) return cudaErrorInvalidValue;
+    if (!get_map(tc, ep.dst, pb.Mp, ep.ld_dst, pb.batch, 128, &mdst)) return cudaErrorInvalidValue;
+    if (ep.aux) {
+      if (ep.bs_aux != pb.Mp * ep.ld_aux) return cudaErrorInvalidValue;
+      if (!get_map(tc, ep.aux, pb.Mp, ep.ld_aux, pb.batch, 128, &maux)) return cudaErrorInvalidValue;
+    }
+    if (ep.dst_t) {
+      if (ep.bs_dst_t != pb.Np * ep.ld_dst_t) return cudaErrorInvalidValue;
+      if (!get_map(tc, ep.dst_t, pb.Np, ep.ld_dst_t, pb.batch, 64, &mdt)) return cudaErrorInvalidValue;
+    }
+  }
   const int64_t mt = pb.Mp / kBM, nt = pb.Np / kBN;
   int64_t per_mat;
   if (pb.symmetric) {
@@ -358,8 +525,9 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   if (total > 0x7fffffffLL) return cudaErrorInvalidValue;
   const int grid = (int)std::min<int64_t>(total, tc->sm_count);
   *launches += 1;
-  gemm_tc_kernel<<<grid, kTcThreads, kSmemBytes, stream>>>(mp, mq, (int)(pb.Kp / kBK), (int)per_mat, (int)total,
-                                                           pb.symmetric, (int)mt, ep, status);
+  gemm_tc_kernel<<<grid, kTcThreads, kSmemBytes, stream>>>(mp, mq, maux, mdst, mdt, (int)(pb.Kp / kBK),
+                                                           (int)per_mat, (int)total, pb.symmetric, (int)mt, ep,
+                                                           status);
   return cudaGetLastError();
 }
 

@@ -3,10 +3,15 @@
 // struct Epilogue (polynomial coefficients, Frobenius scale, mirror write,
 // transposed copy of X, final parameter update).
 //
-// One persistent CTA per SM, 352 threads:
-//   warp 0      TMA producer: 128x64 tile of P and 256x64 tile of Q per stage
-//               (cp.async.bulk.tensor, 128-byte swizzle, no multicast)
-//   warp 1      tcgen05.mma issuer (one lane), owns the TMEM allocation
+// Persistent CTA pairs (clusters of two CTAs on two SMs), 352 threads per CTA.
+// A pair computes a 256x256 tile with tcgen05.mma.cta_group::2: each CTA holds
+// 128 rows of P and 128 of the 256 rows of Q in shared memory, and the
+// accumulator rows of its half in its own tensor memory.
+//   warp 0      TMA producer: 128x64 tile of P and 128x64 tile of Q per stage
+//               (cp.async.bulk.tensor, 128-byte swizzle, no multicast); both
+//               CTAs signal the leader's barrier
+//   warp 1      tcgen05.mma issuer (one lane of the leader CTA); owns the
+//               TMEM allocation of its CTA
 //   warps 2..9  epilogue arithmetic: two warps per TMEM lane quadrant; the
 //               tile is finished in four slabs of 64 columns.  Per slab:
 //               tcgen05.ld of the fp32 accumulator, auxiliary operand read
@@ -34,7 +39,7 @@ constexpr int kBM = 128;          // tile rows  (UMMA M)
 constexpr int kBN = 256;          // tile cols  (UMMA N)
 constexpr int kBK = 64;           // k per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
-constexpr int kStages = 3;
+constexpr int kStages = 5;
 constexpr int kEpiWarps = 8;         // two warps per TMEM lane quadrant
 constexpr int kIoWarp = 2 + kEpiWarps;
 constexpr int kTcThreads = 32 * (kIoWarp + 1);
@@ -44,15 +49,16 @@ constexpr int kEpiBufs = 2;
 constexpr uint32_t kSlabBytes = 128 * kSlabCols * 2;        // result slab, also the aux slab
 constexpr uint32_t kEpiBufBytes = 2 * kSlabBytes;           // + transposed slab (2 boxes of 64x64)
 constexpr uint32_t kBytesA = kBM * kBK * 2;
-constexpr uint32_t kBytesB = kBN * kBK * 2;
+constexpr uint32_t kBytesB = (kBN / 2) * kBK * 2;   // each CTA of the pair holds half of Q's rows
 constexpr uint32_t kStageBytes = kBytesA + kBytesB;
 constexpr uint32_t kTmemCols = 512;
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s
 constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + (size_t)kEpiBufs * kEpiBufBytes + 256;
 
-// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128.
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 256
+// (two CTAs x 128 rows).
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) |
-                            ((uint32_t)(kBM >> 4) << 24);
+                            ((uint32_t)((2 * kBM) >> 4) << 24);
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -106,6 +112,33 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
       : "memory");
 }
+// Load whose completion is counted on the pair leader's barrier (`bar_cluster`
+// is a shared::cluster address).
+__device__ __forceinline__ void tma_load_3d_pair(void* dst, const CUtensorMap* map, uint32_t bar_cluster, int x,
+                                                 int y, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(bar_cluster), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+// shared::cluster address of `p` in the CTA of rank `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_rank(const void* p, uint32_t rank) {
+  uint32_t out;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(smem_u32(p)), "r"(rank));
+  return out;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void tma_store_3d(const void* src, const CUtensorMap* map, int x, int y, int z) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
                ::"l"((uint64_t)map), "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z)
@@ -128,13 +161,19 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
+// Arrives on the barrier at this offset in both CTAs of the pair once all MMAs
+// issued so far have completed.
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+#pragma unroll
+  for (uint32_t r = 0; r < 2; ++r) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(map_to_rank(bar, r))
+                 : "memory");
+  }
 }
 // Issues the TMEM load; the registers are valid after tmem_ld_wait().
 __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
@@ -193,25 +232,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_rank();       // 0 = leader of the pair
   const bool staged = ep.kind == 0;           // product epilogue through shared memory and TMA
   const bool has_aux = ep.aux != nullptr;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], kEpiWarps); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 2 * kEpiWarps); }
     for (int e = 0; e < kEpiBufs; ++e) { mbar_init(&eready[e], 1); mbar_init(&edone[e], kEpiWarps); }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                  "r"(kTmemCols)
                  : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  cluster_sync_all();                         // the peer's barriers are initialised too
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
@@ -227,23 +268,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           const uint32_t ph = (it / kStages) & 1;
           if (!mbar_wait(&empty[s], ph ^ 1, abort_flag, status)) { ok = false; break; }
           uint8_t* sa = smem + (size_t)s * kStageBytes;
-          mbar_expect_tx(&full[s], kStageBytes);
-          tma_load_3d(sa, &mapP, &full[s], kt * kBK, c.ti * kBM, c.b);
-          tma_load_3d(sa + kBytesA, &mapQ, &full[s], kt * kBK, c.tj * kBN, c.b);
+          // The leader's barrier counts the bytes of both CTAs' loads.
+          if (rank == 0) mbar_expect_tx(&full[s], 2 * kStageBytes);
+          const uint32_t lead_full = map_to_rank(&full[s], 0);
+          tma_load_3d_pair(sa, &mapP, lead_full, kt * kBK, c.ti * kBM, c.b);
+          tma_load_3d_pair(sa + kBytesA, &mapQ, lead_full, kt * kBK, c.tj * kBN + (int)rank * (kBN / 2), c.b);
         }
       }
-      // Drain: every load issued must have landed before shared memory is released.
-      const uint32_t n_issued = it;
-      for (uint32_t k = (n_issued > kStages ? n_issued - kStages : 0); k < n_issued; ++k) {
-        const uint64_t t0 = global_ns();
-        while (!mbar_try_wait(&full[k % kStages], (k / kStages) & 1)) {
-          if (global_ns() - t0 > 1000000ull) break;   // 1 ms
+      // Drain: every load issued must have landed before shared memory is
+      // released.  The leader sees the byte counts of both CTAs on its own
+      // barriers; the closing cluster barrier keeps the peer alive until then.
+      if (rank == 0) {
+        const uint32_t n_issued = it;
+        for (uint32_t k = (n_issued > kStages ? n_issued - kStages : 0); k < n_issued; ++k) {
+          const uint64_t t0 = global_ns();
+          while (!mbar_try_wait(&full[k % kStages], (k / kStages) & 1)) {
+            if (global_ns() - t0 > 1000000ull) break;   // 1 ms
+          }
         }
       }
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       uint32_t it = 0, acc_it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_it) {
@@ -264,9 +311,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
             // advance 16 elements = 32 bytes inside the swizzled row: +2 in 16-byte units
             umma_bf16(tacc, da + 2 * k, db + 2 * k, (kt | k) != 0);
           }
-          umma_commit(&empty[s]);        // frees the stage when these MMAs have read it
+          umma_commit_pair(&empty[s]);        // frees the stage in both CTAs when these MMAs have read it
         }
-        if (ok) umma_commit(&tfull[a]);  // accumulator complete
+        if (ok) umma_commit_pair(&tfull[a]);  // accumulator complete in both CTAs
       }
     }
   } else if (warp == kIoWarp) {
@@ -411,16 +458,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty[a]);
+      if (lane == 0) mbar_arrive_cluster(map_to_rank(&tempty[a], 0));   // the leader issues the MMAs
     }
   }
 
   // ---------------------------------------------------------------- teardown
+  // Neither CTA may leave while its partner can still touch its shared
+  // memory, barriers or tensor memory.
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  cluster_sync_all();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -434,6 +484,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 struct TcContext {
   EncodeTiledFn encode = nullptr;
   int sm_count = 0;
+  int max_pairs = 0;   // CTA pairs that can be resident at once
   std::map<std::tuple<const void*, int64_t, int64_t, int, int>, CUtensorMap> cache;
 };
 
@@ -467,6 +518,25 @@ TcContext* tc_create(std::string* err) {
     delete tc;
     return nullptr;
   }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(tc->sm_count & ~1, 1, 1);
+  cfg.blockDim = dim3(kTcThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n_clusters = 0;
+  ce = cudaOccupancyMaxActiveClusters(&n_clusters, gemm_tc_kernel, &cfg);
+  if (ce != cudaSuccess || n_clusters < 1) {
+    if (err) *err = std::string("cudaOccupancyMaxActiveClusters: ") + cudaGetErrorString(ce);
+    delete tc;
+    return nullptr;
+  }
+  tc->max_pairs = n_clusters;
   return tc;
 }
 
@@ -497,7 +567,7 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   if (pb.Mp % kBN != 0 || pb.Np % kBN != 0 || pb.Kp % kBK != 0) return cudaErrorInvalidValue;
   CUtensorMap mp, mq, maux, mdst, mdt;
   if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
-  if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN, &mq)) return cudaErrorInvalidValue;
+  if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
   // Epilogue maps (product epilogues only): auxiliary and result slabs of 128
   // rows x 64 columns, transposed result in boxes of 64 x 64.
   maux = mp; mdst = mp; mdt = mp;
@@ -523,12 +593,23 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   }
   const int64_t total = per_mat * pb.batch;
   if (total > 0x7fffffffLL) return cudaErrorInvalidValue;
-  const int grid = (int)std::min<int64_t>(total, tc->sm_count);
+  // total is even: CTA 2p and 2p+1 (one cluster) take the two 128-row halves of a 256x256 tile.
+  const int pairs = (int)std::min<int64_t>(total / 2, tc->max_pairs);
   *launches += 1;
-  gemm_tc_kernel<<<grid, kTcThreads, kSmemBytes, stream>>>(mp, mq, maux, mdst, mdt, (int)(pb.Kp / kBK),
-                                                           (int)per_mat, (int)total, pb.symmetric, (int)mt, ep,
-                                                           status);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(kTcThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel, mp, mq, maux, mdst, mdt, (int)(pb.Kp / kBK), (int)per_mat,
+                            (int)total, pb.symmetric, (int)mt, ep, status);
 }
 
 }  // namespace prm

@@ -328,6 +328,8 @@ def main():
         "refresh_steps_timed": n_ref, "row_steps_timed": n_row,
         "gpu_launches": launches,
         "clocks": clocks,
+        # device time per kernel class over the whole timed region (CUDA events inside the library)
+        "kernel_classes": {k: {"ms": round(v[0], 3), "launches": v[1]} for k, v in prof.items()},
     }
     if n_row:
         gbs = row_bytes / (mean_row * 1e-3) / 1e9

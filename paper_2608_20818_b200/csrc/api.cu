@@ -28,10 +28,11 @@ struct prm_ctx {
   std::vector<int> group_of_mat, order_in_group, slot_of_mat;   // slot = index in pointer tables
 
   // workspace layout (byte offsets)
-  size_t off_status = 0, off_tables = 0, off_fro = 0, off_alpha = 0, off_ns = 0, total_bytes = 0;
+  size_t off_status = 0, off_tables = 0, off_pmaps = 0, off_fro = 0, off_alpha = 0, off_ns = 0, total_bytes = 0;
   char* ws = nullptr;
   size_t ws_bytes = 0;
   std::vector<void*> host_tables;   // 3*n_mats, grouped order: params | grads | momentum
+  std::vector<unsigned char> host_pmaps;   // n_mats tensor maps of 128 bytes over the parameters (table order)
   bool tables_uploaded = false;
 
   TcContext* tc = nullptr;
@@ -92,6 +93,7 @@ static void compute_layout(prm_ctx* c) {
   size_t off = 0;
   c->off_status = off; off += 256;
   c->off_tables = off; off = align_up(off + (size_t)3 * c->n_mats * sizeof(void*), 256);
+  c->off_pmaps = off;  off = align_up(off + (size_t)128 * c->n_mats, 256);
   size_t fro_max = 0, ns_max = 0;
   int batch_max = 1;
   for (Group& g : c->groups) {
@@ -157,6 +159,7 @@ extern "C" int prm_create(prm_ctx** out, const int64_t* shapes, int n_mats, int 
   for (int i = 0; i < n_mats; ++i)
     c->slot_of_mat[i] = c->groups[c->group_of_mat[i]].first + c->order_in_group[i];
   c->host_tables.assign((size_t)3 * n_mats, nullptr);
+  c->host_pmaps.assign((size_t)128 * n_mats, 0);
   compute_layout(c);
   *out = c;
   return PRM_OK;
@@ -283,6 +286,8 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
         eu.kind = 1; eu.tables = t; eu.first = first;
         eu.rows = (int)g.rows; eu.cols = (int)g.cols; eu.tall = g.tall ? 1 : 0;
         eu.io_fp32 = c->io_fp32; eu.decay = s.decay; eu.lr_s = s.lr_s;
+        // bf16 parameters with 16-byte aligned rows are updated through TMA-staged tiles.
+        if (!c->check_mode && !c->io_fp32 && g.cols % 8 == 0) eu.param_maps = c->ws + c->off_pmaps;
       }
       if ((ce = gemm(pu, eu, it + 1 < kNsIters ? PRM_PROF_UPDATE : PRM_PROF_UPDATE_FINAL)) != cudaSuccess) break;
       cur ^= 1;
@@ -317,6 +322,17 @@ static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
     ce = cudaMemcpyAsync(c->ws + c->off_tables, c->host_tables.data(), (size_t)3 * n * sizeof(void*),
                          cudaMemcpyHostToDevice, stream);
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("pointer tables: ") + cudaGetErrorString(ce));
+    if (!c->check_mode && !c->io_fp32) {
+      for (int i = 0; i < n; ++i) {
+        const Group& g = c->groups[c->group_of_mat[i]];
+        if (g.cols % 8 != 0) continue;
+        if (!tc_encode_param_map(c->tc, params[i], g.rows, g.cols, g.tall ? 1 : 0,
+                                 c->host_pmaps.data() + (size_t)128 * c->slot_of_mat[i]))
+          return fail(c, PRM_ERR_CUDA, "cannot encode a tensor map over a parameter matrix");
+      }
+      ce = cudaMemcpyAsync(c->ws + c->off_pmaps, c->host_pmaps.data(), (size_t)128 * n, cudaMemcpyHostToDevice, stream);
+      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("parameter tensor maps: ") + cudaGetErrorString(ce));
+    }
     c->tables_uploaded = true;
   }
   if (grads_host) {

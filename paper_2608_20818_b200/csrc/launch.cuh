@@ -31,6 +31,9 @@ struct Epilogue {
   int tall = 0;
   int io_fp32 = 0;
   float decay = 1.f, lr_s = 0.f;
+  // Tensor-core path only: device array of 128-byte tensor maps over the
+  // parameter matrices (table order); null selects per-thread accesses.
+  const void* param_maps = nullptr;
 };
 
 // One batched product.  P: [batch][Mp][Kp], Q: [batch][Np][Kp]; Mp, Np, Kp
@@ -65,6 +68,7 @@ cudaError_t launch_gemm_simt(const GemmProblem& pb, const Epilogue& ep, cudaStre
 struct TcContext;
 cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue& ep, int* status,
                            cudaStream_t stream, int64_t* launches);
+bool tc_encode_param_map(TcContext* tc, const void* base, int64_t rows, int64_t cols, int tall, void* out128);
 TcContext* tc_create(std::string* err);
 void tc_destroy(TcContext* tc);
 

@@ -19,12 +19,18 @@
 //               transposed, into a second slab
 //   warp 10     epilogue I/O: TMA load of the auxiliary slab, TMA stores of
 //               the result slab and of its transpose
-// All global traffic of the product epilogues therefore moves as 128-byte
-// swizzled TMA boxes; per-thread global accesses remain only in the final
-// parameter update.  Two 256-column accumulators in TMEM let the epilogue of
-// tile n overlap the main loop of tile n+1.  Every mbarrier wait is bounded:
-// on expiry the CTA raises the status word, drains and exits cleanly.
+// All global traffic of the epilogues therefore moves as 128-byte swizzled
+// TMA boxes, the final parameter update included (the parameter tile is loaded
+// into the second slab, updated there and stored back; tall matrices use the
+// transposed boxes).  Per-thread global accesses remain only for fp32
+// parameters and for column counts that are not a multiple of 8.  Two
+// 256-column accumulators in TMEM let the epilogue of tile n overlap the main
+// loop of tile n+1.  Every mbarrier wait is bounded: on expiry the CTA raises
+// the status word, drains and exits cleanly.
 #include <cuda.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
 
 #include <map>
 #include <tuple>
@@ -111,6 +117,17 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, u
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y), "r"(z)
       : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const void* src, const CUtensorMap* map, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"((uint64_t)map), "r"(smem_u32(src)), "r"(x), "r"(y)
+               : "memory");
 }
 // Load whose completion is counted on the pair leader's barrier (`bar_cluster`
 // is a shared::cluster address).
@@ -233,8 +250,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_rank();       // 0 = leader of the pair
-  const bool staged = ep.kind == 0;           // product epilogue through shared memory and TMA
+  // fin: final parameter update with the parameter tile staged through shared
+  // memory (per-matrix tensor maps in global memory); otherwise kind 1 falls
+  // back to per-thread global accesses.
+  const bool fin = ep.kind == 1 && ep.param_maps != nullptr;
+  const bool staged = ep.kind == 0 || fin;    // epilogue through shared memory and TMA
   const bool has_aux = ep.aux != nullptr;
+  const CUtensorMap* pmaps = reinterpret_cast<const CUtensorMap*>(ep.param_maps);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -327,11 +349,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
       const uint32_t n_slabs = (uint32_t)n_my_tiles * kSlabs;
       auto prepare = [&](uint32_t g) {
         const int bsel = g % kEpiBufs;
-        if (has_aux) {
+        if (has_aux || fin) {
           const TileCoord c = decode_tile(blockIdx.x + (int)(g / kSlabs) * gridDim.x, tiles_per_mat, symmetric, mt);
-          mbar_expect_tx(&eready[bsel], kSlabBytes);
-          tma_load_3d(ebuf + (size_t)bsel * kEpiBufBytes, &mapAux, &eready[bsel],
-                      c.tj * kBN + (int)(g % kSlabs) * kSlabCols, c.ti * kBM, c.b);
+          const int j0 = c.tj * kBN + (int)(g % kSlabs) * kSlabCols;
+          uint8_t* buf = ebuf + (size_t)bsel * kEpiBufBytes;
+          mbar_expect_tx(&eready[bsel], (has_aux ? kSlabBytes : 0u) + (fin ? kSlabBytes : 0u));
+          if (has_aux) tma_load_3d(buf, &mapAux, &eready[bsel], j0, c.ti * kBM, c.b);
+          if (fin) {
+            // Parameter tile into the second slab: as stored (wide), or the
+            // transposed region in two 64x64 boxes (tall).  Out-of-range parts read as zero.
+            const CUtensorMap* pm = pmaps + ep.first + c.b;
+            if (!ep.tall) {
+              tma_load_2d(buf + kSlabBytes, pm, &eready[bsel], j0, c.ti * kBM);
+            } else {
+              tma_load_2d(buf + kSlabBytes, pm, &eready[bsel], c.ti * kBM, j0);
+              tma_load_2d(buf + kSlabBytes + kSlabBytes / 2, pm, &eready[bsel], c.ti * kBM + 64, j0);
+            }
+          }
         } else {
           mbar_arrive(&eready[bsel]);
         }
@@ -343,10 +377,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
         const TileCoord c = decode_tile(blockIdx.x + (int)(g / kSlabs) * gridDim.x, tiles_per_mat, symmetric, mt);
         const int j0 = c.tj * kBN + (int)(g % kSlabs) * kSlabCols;
         const uint8_t* buf = ebuf + (size_t)bsel * kEpiBufBytes;
-        tma_store_3d(buf, &mapDst, j0, c.ti * kBM, c.b);
-        if (c.mirror && ep.dst_t != nullptr) {
-          tma_store_3d(buf + kSlabBytes, &mapDstT, c.ti * kBM, j0, c.b);
-          tma_store_3d(buf + kSlabBytes + kSlabBytes / 2, &mapDstT, c.ti * kBM + 64, j0, c.b);
+        if (fin) {
+          const CUtensorMap* pm = pmaps + ep.first + c.b;
+          if (!ep.tall) {
+            tma_store_2d(buf + kSlabBytes, pm, j0, c.ti * kBM);
+          } else {
+            tma_store_2d(buf + kSlabBytes, pm, c.ti * kBM, j0);
+            tma_store_2d(buf + kSlabBytes + kSlabBytes / 2, pm, c.ti * kBM + 64, j0);
+          }
+        } else {
+          tma_store_3d(buf, &mapDst, j0, c.ti * kBM, c.b);
+          if (c.mirror && ep.dst_t != nullptr) {
+            tma_store_3d(buf + kSlabBytes, &mapDstT, c.ti * kBM, j0, c.b);
+            tma_store_3d(buf + kSlabBytes + kSlabBytes / 2, &mapDstT, c.ti * kBM + 64, j0, c.b);
+          }
         }
         tma_store_commit();
         if (g + kEpiBufs < n_slabs) {
@@ -355,7 +399,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
         }
       }
       tma_store_wait_all();
-      if (has_aux) {
+      if (has_aux || fin) {
         // Drain auxiliary loads that were issued but never consumed (abort path only).
         for (int e = 0; e < kEpiBufs; ++e) {
           const uint64_t t0 = global_ns();
@@ -414,6 +458,31 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
             } else {
 #pragma unroll
               for (int k = 0; k < 8; ++k) x[k] = 0.f;
+            }
+            if (fin) {
+              // W <- decay*W - lr*s*X_5 on the staged parameter tile.
+              if (!ep.tall) {
+                int4* pp = reinterpret_cast<int4*>(buf + kSlabBytes + sw128(row, half * 4 + v));
+                int4 pw = *pp;
+                __nv_bfloat162* w2 = reinterpret_cast<__nv_bfloat162*>(&pw);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const float2 w = __bfloat1622float2(w2[k]);
+                  const float v0 = ka * __uint_as_float(r[8 * v + 2 * k]) + kx * x[2 * k];
+                  const float v1 = ka * __uint_as_float(r[8 * v + 2 * k + 1]) + kx * x[2 * k + 1];
+                  w2[k] = __floats2bfloat162_rn(ep.decay * w.x - ep.lr_s * v0, ep.decay * w.y - ep.lr_s * v1);
+                }
+                *pp = pw;
+              } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                  const uint32_t cc = half * 32 + v * 8 + k;
+                  __nv_bfloat16* pe = reinterpret_cast<__nv_bfloat16*>(tbuf + sw128(cc, rt >> 3) + (rt & 7) * 2);
+                  const float vk = ka * __uint_as_float(r[8 * v + k]) + kx * x[k];
+                  *pe = __float2bfloat16_rn(ep.decay * __bfloat162float(*pe) - ep.lr_s * vk);
+                }
+              }
+              continue;
             }
             int4 outv;
             __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&outv);
@@ -537,6 +606,7 @@ TcContext* tc_create(std::string* err) {
     return nullptr;
   }
   tc->max_pairs = n_clusters;
+  if (getenv("PRM_VERBOSE")) fprintf(stderr, "prm: %d SMs, %d resident CTA pairs\n", tc->sm_count, n_clusters);
   return tc;
 }
 
@@ -561,6 +631,25 @@ static bool get_map(TcContext* tc, const void* base, int64_t rows, int64_t kdim,
   return true;
 }
 
+// Tensor map over one bf16 parameter matrix (rows x cols, row-major) for the
+// staged final update: boxes of 128 rows x 64 columns for wide matrices, of
+// 64 x 64 for tall ones (whose tile is written transposed).  out128 receives
+// the 128-byte descriptor.  Needs cols % 8 == 0 and a 16-byte aligned base.
+bool tc_encode_param_map(TcContext* tc, const void* base, int64_t rows, int64_t cols, int tall, void* out128) {
+  if (!tc || (cols % 8) != 0 || ((uintptr_t)base & 15) != 0) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64, tall ? 64u : 128u};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMap m;
+  CUresult r = tc->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  memcpy(out128, &m, sizeof(CUtensorMap));
+  return true;
+}
+
 cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue& ep, int* status,
                            cudaStream_t stream, int64_t* launches) {
   if (!tc) return cudaErrorInvalidValue;
@@ -571,13 +660,13 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   // Epilogue maps (product epilogues only): auxiliary and result slabs of 128
   // rows x 64 columns, transposed result in boxes of 64 x 64.
   maux = mp; mdst = mp; mdt = mp;
+  if (ep.aux && (ep.kind == 0 || ep.param_maps)) {
+    if (ep.bs_aux != pb.Mp * ep.ld_aux) return cudaErrorInvalidValue;
+    if (!get_map(tc, ep.aux, pb.Mp, ep.ld_aux, pb.batch, 128, &maux)) return cudaErrorInvalidValue;
+  }
   if (ep.kind == 0) {
     if (ep.bs_dst != pb.Mp * ep.ld_dst) return cudaErrorInvalidValue;
     if (!get_map(tc, ep.dst, pb.Mp, ep.ld_dst, pb.batch, 128, &mdst)) return cudaErrorInvalidValue;
-    if (ep.aux) {
-      if (ep.bs_aux != pb.Mp * ep.ld_aux) return cudaErrorInvalidValue;
-      if (!get_map(tc, ep.aux, pb.Mp, ep.ld_aux, pb.batch, 128, &maux)) return cudaErrorInvalidValue;
-    }
     if (ep.dst_t) {
       if (ep.bs_dst_t != pb.Np * ep.ld_dst_t) return cudaErrorInvalidValue;
       if (!get_map(tc, ep.dst_t, pb.Np, ep.ld_dst_t, pb.batch, 64, &mdt)) return cudaErrorInvalidValue;

@@ -20,13 +20,14 @@ namespace prm {
 constexpr int kRowThreads = 256;
 
 // ------------------------------------------------------------------ wide
-// One row per cluster of CLUSTER CTAs; each thread keeps VPT vectors of 8
-// elements of U in registers between the reduction and the update, so every
-// byte crosses HBM once: 14 B/element with bf16 I/O.
-template <typename IO, int VPT, int CLUSTER>
-__global__ void __launch_bounds__(kRowThreads)
+// One row per CTA of THREADS threads (or per cluster of CLUSTER CTAs for very
+// long rows); each thread keeps VPT vectors of 8 elements of U in registers
+// between the reduction and the update, so every byte crosses HBM once:
+// 14 B/element with bf16 I/O.
+template <typename IO, int VPT, int CLUSTER, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
-  __shared__ float warp_part[kRowThreads / 32];
+  __shared__ float warp_part[THREADS / 32];
   __shared__ float cta_part;
 
   const int rank = CLUSTER > 1 ? (int)cg::this_cluster().block_rank() : 0;
@@ -48,7 +49,7 @@ rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
   float acc = 0.f;
 #pragma unroll
   for (int k = 0; k < VPT; ++k) {
-    const int v = v_begin + threadIdx.x + k * kRowThreads;
+    const int v = v_begin + threadIdx.x + k * THREADS;
     if (v < v_end) {
       float gv[8], mv[8];
       load8_stream(g + 8 * v, gv);
@@ -70,7 +71,7 @@ rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
   __syncthreads();
   float total = 0.f;
 #pragma unroll
-  for (int w = 0; w < kRowThreads / 32; ++w) total += warp_part[w];
+  for (int w = 0; w < THREADS / 32; ++w) total += warp_part[w];
   if constexpr (CLUSTER > 1) {
     cg::cluster_group cluster = cg::this_cluster();
     if (threadIdx.x == 0) cta_part = total;
@@ -84,7 +85,7 @@ rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
   const float coef = s.lr_s * s.gamma / nu;
 #pragma unroll
   for (int k = 0; k < VPT; ++k) {
-    const int v = v_begin + threadIdx.x + k * kRowThreads;
+    const int v = v_begin + threadIdx.x + k * THREADS;
     if (v < v_end) {
       float pf[8];
       pv[k].get(pf);
@@ -245,13 +246,13 @@ rowstep_tall_pass2_kernel(PtrTables t, int first, int rows, int cols, StepScalar
 }
 
 // --------------------------------------------------------------- launchers
-template <typename IO, int VPT, int CLUSTER>
+template <typename IO, int VPT, int CLUSTER, int THREADS = kRowThreads>
 static cudaError_t launch_wide_inst(const PtrTables& t, const Group& g, const StepScalars& s,
                                     cudaStream_t stream) {
   const int64_t nrows = (int64_t)g.count * g.rows;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(nrows * CLUSTER), 1, 1);
-  cfg.blockDim = dim3(kRowThreads, 1, 1);
+  cfg.blockDim = dim3(THREADS, 1, 1);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -260,7 +261,7 @@ static cudaError_t launch_wide_inst(const PtrTables& t, const Group& g, const St
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, rowstep_wide_kernel<IO, VPT, CLUSTER>, t, g.first, (int)g.rows,
+  return cudaLaunchKernelEx(&cfg, rowstep_wide_kernel<IO, VPT, CLUSTER, THREADS>, t, g.first, (int)g.rows,
                             (int)g.cols, s);
 }
 
@@ -276,11 +277,15 @@ static cudaError_t launch_wide(const PtrTables& t, const Group& g, const StepSca
         t, g.first, (int)g.rows, (int)g.cols, s);
     return cudaGetLastError();
   }
+  // Rows up to 32768 elements stay inside one CTA (wider CTAs for longer
+  // rows): measured faster than splitting a row over a cluster, whose two
+  // cluster barriers cost more than the lower occupancy.
   if (cols <= 2048) return launch_wide_inst<IO, 1, 1>(t, g, s, stream);
   if (cols <= 4096) return launch_wide_inst<IO, 2, 1>(t, g, s, stream);
-  if (cols <= 8192) return launch_wide_inst<IO, 4, 1>(t, g, s, stream);
-  if (cols <= 16384) return launch_wide_inst<IO, 4, 2>(t, g, s, stream);
-  if (cols <= 32768) return launch_wide_inst<IO, 4, 4>(t, g, s, stream);
+  if (cols <= 8192) return launch_wide_inst<IO, 2, 1, 512>(t, g, s, stream);
+  if (cols <= 16384) return launch_wide_inst<IO, 4, 1, 512>(t, g, s, stream);
+  if (cols <= 24576) return launch_wide_inst<IO, 3, 1, 1024>(t, g, s, stream);
+  if (cols <= 32768) return launch_wide_inst<IO, 4, 2, 512>(t, g, s, stream);
   return launch_wide_inst<IO, 4, 8>(t, g, s, stream);
 }
 

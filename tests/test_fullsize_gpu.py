@@ -1,0 +1,145 @@
+"""Parity at the benchmark's full sizes, in the launch configuration that
+bench.py times (one handle over the whole shape set, default options).
+
+The oracle cannot run every matrix of these shape sets, so each case checks
+  * the row step on sampled stored rows (wide) and stored columns (tall) of
+    sampled matrices against the oracle, element by element;
+  * the refresh on one whole block (one matrix of every shape): tensor-core
+    result against the fp32 check mode for all five shapes, and against the
+    fp64 oracle (all five shapes; the square one only for configuration 5).
+Configuration 5 needs 181 GB for its 48 blocks; it runs here with 8 blocks
+(the blocks are identical and independent).
+"""
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import prm_oracle as O
+from paper_2608_20818_b200 import binding as B
+from paper_2608_20818_b200.workloads import make_grad, make_momentum, make_param, workload
+from tests import util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_cfg(wl):
+    return O.OracleConfig(K=wl.K, beta=wl.beta, nesterov=wl.nesterov, lr=wl.lr, wd=wl.wd, gamma=wl.gamma)
+
+
+def _check_row_step_samples(wl, idx, W0, M0, G, W1, M1, rng):
+    """Sampled rows (wide) or columns (tall) of matrix idx against the oracle."""
+    cfg = _oracle_cfg(wl)
+    m, n = wl.shapes[idx]
+    s = O.shape_scale(m, n, cfg.scale_mode)
+    decay = 1.0 - cfg.lr * cfg.wd
+    if m <= n:
+        rows = rng.choice(m, size=8, replace=False)
+        for r in rows:
+            w0, m0, g = (U.to_np64(x[r:r + 1]) for x in (W0, M0, G))
+            mt = O.momentum_update(m0, g, cfg.beta)
+            u = O.direction_input(mt, g, cfg.beta, cfg.nesterov)
+            want = decay * w0 - cfg.lr * s * cfg.gamma * O.rownorm(u, cfg.eps_row)
+            U.assert_elementwise(U.to_np64(M1[r:r + 1]), mt, False, f"momentum row {r} of {idx}")
+            U.assert_elementwise(U.to_np64(W1[r:r + 1]), want, True, f"param row {r} of {idx}")
+    else:
+        cols = rng.choice(n, size=8, replace=False)
+        for c in cols:
+            w0, m0, g = (U.to_np64(x[:, c:c + 1]).T for x in (W0, M0, G))     # 1 x m oriented rows
+            mt = O.momentum_update(m0, g, cfg.beta)
+            u = O.direction_input(mt, g, cfg.beta, cfg.nesterov)
+            want = decay * w0 - cfg.lr * s * cfg.gamma * O.rownorm(u, cfg.eps_row)
+            U.assert_elementwise(U.to_np64(M1[:, c:c + 1]).T, mt, False, f"momentum col {c} of {idx}")
+            U.assert_elementwise(U.to_np64(W1[:, c:c + 1]).T, want, True, f"param col {c} of {idx}")
+
+
+def _run_config(config_id, blocks, oracle_shapes):
+    wl = workload(config_id, blocks)
+    n = len(wl.shapes)
+    dev = "cuda"
+    rng = np.random.default_rng(config_id)
+    params = [make_param(wl, i, dev) for i in range(n)]
+    moms = [make_momentum(wl, i, dev) for i in range(n)]
+    grads = [make_grad(wl, i, 0, dev) for i in range(n)]
+    opt = B.PeriodicRowwiseMuon(wl.shapes, wl.K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma)
+    block = int(rng.integers(0, n // 5))
+    sample = list(range(5 * block, 5 * block + 5))            # one matrix of every shape
+
+    # ---- row step (t = 1), from momentum made non-zero by a first row step (t = 2 of another period)
+    opt.step(params, grads, moms, 2)
+    pre = {i: (params[i].clone(), moms[i].clone()) for i in sample}
+    opt.step(params, grads, moms, 1)
+    torch.cuda.synchronize()
+    assert opt.status() == B.PRM_OK
+    for i in sample:
+        _check_row_step_samples(wl, i, pre[i][0], pre[i][1], grads[i], params[i], moms[i], rng)
+
+    # ---- refresh (t = K).  The sampled block starts from zero parameters, so the step writes
+    # -lr*s*NS5(U) and the bf16 store keeps 2^-9 relative precision on the direction itself.
+    for i in sample:
+        params[i].zero_()
+    pre = {i: moms[i].clone() for i in sample}
+    opt.step(params, grads, moms, wl.K)
+    torch.cuda.synchronize()
+    assert opt.status() == B.PRM_OK
+    # the same five matrices through the fp32 check mode
+    shapes5 = [wl.shapes[i] for i in sample]
+    chk = B.PeriodicRowwiseMuon(shapes5, wl.K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma, check_mode=True)
+    Wc = [torch.zeros_like(params[i]) for i in sample]
+    Mc = [pre[i].clone() for i in sample]
+    chk.step(Wc, [grads[i] for i in sample], Mc, wl.K)
+    torch.cuda.synchronize()
+    assert chk.status() == B.PRM_OK
+    cfg = _oracle_cfg(wl)
+    out = {}
+    for k, i in enumerate(sample):
+        assert torch.equal(Mc[k], moms[i]), "momentum must not depend on the NS5 mode"
+        d_fast, d_chk = params[i].double(), Wc[k].double()
+        assert float(d_chk.abs().max()) > 0
+        err = float(torch.linalg.norm(d_fast - d_chk) / torch.linalg.norm(d_chk))
+        out[wl.shapes[i]] = err
+        assert err <= 2e-2, (wl.shapes[i], err)
+        if wl.shapes[i] in oracle_shapes:
+            Wr, Mr = O.step_matrix(np.zeros(wl.shapes[i]), U.to_np64(grads[i]), U.to_np64(pre[i]), wl.K, cfg)
+            U.assert_elementwise(U.to_np64(moms[i]), Mr, False, f"momentum {wl.shapes[i]}")
+            e_fast = U.rel_fro(U.to_np64(params[i]), Wr)
+            e_chk = U.rel_fro(U.to_np64(Wc[k]), Wr)
+            assert e_fast <= 2e-2, (wl.shapes[i], e_fast)
+            assert e_chk <= 4e-3, (wl.shapes[i], e_chk)       # fp32 arithmetic, bf16 store (2^-9)
+    opt.close()
+    chk.close()
+    return out
+
+
+def _all_shapes(d):
+    return {(d, 3 * d), (d, d), (d, 4 * d), (4 * d, d), (d, 6 * d)}
+
+
+def test_config2_full():
+    _run_config(2, None, _all_shapes(2048))
+
+
+def test_config3_full():
+    _run_config(3, None, _all_shapes(3072))
+
+
+def test_config4_full():
+    _run_config(4, None, _all_shapes(4096))
+
+
+def test_config5_heavy_tailed_rows_8_blocks():
+    _run_config(5, 8, {(5120, 5120)})
+
+
+def test_check_mode_direction_at_4096():
+    """fp32 check mode against the oracle at d = 4096 with fp32 parameters
+    (W = 0, lr = 1: the step writes the direction itself)."""
+    shapes = [(4096, 4096)]
+    cfg = U.oracle_cfg(K=1, beta=0.95, nesterov=True, lr=1.0, wd=0.0, scale_mode=0)
+    W, G, M = U.make_inputs(shapes, 4096, "fp32", grad_std=1e-3, mom_std=1e-3)
+    W[0].zero_()
+    for mode, tol in ((True, 1e-4), (False, 2e-2)):
+        Wg, _ = U.gpu_step(shapes, W, G, M, 0, cfg, "fp32", mode)
+        Wr, _ = O.step_matrix(U.to_np64(W[0]), U.to_np64(G[0]), U.to_np64(M[0]), 0, cfg)
+        err = U.rel_fro(Wg[0], Wr)
+        assert err <= tol, (mode, err)

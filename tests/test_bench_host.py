@@ -1,0 +1,74 @@
+"""Host-side logic of bench.py: flop and byte accounting, and the N > 1 path
+(independent replicas; the only cross-rank traffic is the max over ranks of
+the timings), exercised with two gloo ranks on CPU."""
+
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as td
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+import bench  # noqa: E402
+from paper_2608_20818_b200.workloads import workload  # noqa: E402
+
+
+def test_accounting_matches_the_shape_sets():
+    # per block: 18 d^2 elements; executed flop 15 r^2 c + 5 r^3, model 20 r^2 c + 10 r^3
+    for cfg, d, blocks in ((2, 2048, 24), (3, 3072, 36), (4, 4096, 42), (5, 5120, 48)):
+        wl = workload(cfg)
+        assert len(wl.shapes) == 5 * blocks
+        assert bench.elements(wl.shapes) == 18 * d * d * blocks
+        ex, mo = bench.ns5_flops(wl.shapes)
+        assert mo == 410 * d ** 3 * blocks          # 70 + 30 + 90 + 90 + 130 per block
+        assert ex == 295 * d ** 3 * blocks          # 50 + 20 + 65 + 65 + 95 per block
+    ex, mo = bench.ns5_flops(workload(4).shapes)
+    assert abs(ex / 1e12 - 851.4) < 0.1 and abs(mo / 1e12 - 1183.3) < 0.1
+    assert abs(14 * bench.elements(workload(4).shapes) / 1e9 - 177.6) < 0.1
+
+
+def _rank_main(rank, world, port, q):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    td.init_process_group("gloo", rank=rank, world_size=world)
+    got = bench.max_over_ranks([1.0 + rank, 10.0 - rank, 5.0])
+    td.barrier()
+    td.destroy_process_group()
+    q.put((rank, got))
+
+
+def test_max_over_ranks_two_gloo_ranks():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 29500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_rank_main, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    out = dict(q.get(timeout=120) for _ in range(2))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert out[0] == out[1] == [2.0, 10.0, 5.0]
+    assert bench.per_replica_ms(100.0, 2) == 50.0
+    assert bench.max_over_ranks([3.0]) == [3.0]          # not distributed: identity
+
+
+def test_reference_arm_runs_on_rank_zero_only():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", OMP_NUM_THREADS="2")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0 and r.stdout.strip() == ""
+    env["RANK"] = "0"
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                        "--steps", "1", "--warmup", "0", "--config", "2"], env=env, capture_output=True, text=True,
+                       timeout=600)
+    assert r.returncode == 0, r.stderr[-500:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "ms/step" and line["higher_is_better"] is False
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
+    assert line["value"] > 0

@@ -33,6 +33,11 @@ from paper_2608_20818_b200.workloads import make_grad, make_momentum, make_param
 METRIC = "amortised optimizer ms/step at K"
 NOMINAL_HBM_GBS = 8000.0       # nominal figure the targets are quoted against
 NOMINAL_BF16_TFLOPS = 2250.0
+# DRAM traffic of the kernels, from ncu captures of a one-block case of the 9B-class set
+# (profiles/gemm_tc_kernel_dit-9b-class_1block.md, profiles/rowstep_kernels_dit-9b-class_1block.md),
+# scaled to a full launch by the work it processes (traffic grows in proportion to it).
+GEMM_DRAM_BYTES_PER_EXEC_FLOP = 784.2e6 / (3 * 4096 ** 2 * 12288 + 4096 ** 3)   # gram + poly + update of one matrix
+ROW_DRAM_BYTES_PER_ELEMENT = 14.0   # wide; the captures never exceed the algorithmic bytes
 
 
 # ----------------------------------------------------------------- accounting
@@ -367,13 +372,17 @@ def main():
         else:
             peak = pk["bf16_tflops_sustained"]
             out["roofline"] = {"bound": "tensor", "achieved": tf_exec, "peak": peak, "unit": "TFLOP/s",
-                               "frac": tf_exec / peak, "traffic": None, "kernel": "gemm_tc_kernel",
+                               "frac": tf_exec / peak,
+                               "traffic": GEMM_DRAM_BYTES_PER_EXEC_FLOP * ex * n_ref / max(1, gemm_launches),
+                               "traffic_unit": "DRAM bytes per launch, scaled from a one-block ncu capture",
+                               "kernel": "gemm_tc_kernel",
                                "launches": gemm_launches, "avg_launch_ms": gemm_ms / max(1, gemm_launches),
                                "peak_source": "%s sustained bf16 matmul" % pk["source"]}
     elif n_row:
         gbs = row_bytes / (row_kernel_ms / n_row * 1e-3) / 1e9
         out["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                           "frac": gbs / pk["hbm_gbs"], "traffic": None, "kernel": "rowstep_*",
+                           "frac": gbs / pk["hbm_gbs"], "traffic": ROW_DRAM_BYTES_PER_ELEMENT * el,
+                           "traffic_unit": "DRAM bytes per row step", "kernel": "rowstep_*",
                            "peak_source": "%s copy bandwidth" % pk["source"]}
     out["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:

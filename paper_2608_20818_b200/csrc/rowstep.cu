@@ -23,9 +23,11 @@ constexpr int kRowThreads = 256;
 // One row per CTA of THREADS threads (or per cluster of CLUSTER CTAs for very
 // long rows); each thread keeps VPT vectors of 8 elements of U in registers
 // between the reduction and the update, so every byte crosses HBM once:
-// 14 B/element with bf16 I/O.
-template <typename IO, int VPT, int CLUSTER, int THREADS>
-__global__ void __launch_bounds__(THREADS)
+// 14 B/element with bf16 I/O.  PREP loads the parameters before the
+// reduction (more registers, fewer resident CTAs); MINB is the number of CTAs
+// per SM the register allocation must allow.
+template <typename IO, int VPT, int CLUSTER, int THREADS, bool PREP = true, int MINB = 1>
+__global__ void __launch_bounds__(THREADS, MINB)
 rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
   __shared__ float warp_part[THREADS / 32];
   __shared__ float cta_part;
@@ -54,7 +56,7 @@ rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
       float gv[8], mv[8];
       load8_stream(g + 8 * v, gv);
       load8_stream(m + 8 * v, mv);
-      pv[k].load_stream(p + 8 * v);
+      if (PREP) pv[k].load_stream(p + 8 * v);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const float mn = s.beta * mv[e] + s.omb * gv[e];
@@ -83,6 +85,13 @@ rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
   }
   const float nu = fmaxf(sqrtf(total), s.eps_row);
   const float coef = s.lr_s * s.gamma / nu;
+  if (!PREP) {
+#pragma unroll
+    for (int k = 0; k < VPT; ++k) {
+      const int v = v_begin + threadIdx.x + k * THREADS;
+      if (v < v_end) pv[k].load_stream(p + 8 * v);
+    }
+  }
 #pragma unroll
   for (int k = 0; k < VPT; ++k) {
     const int v = v_begin + threadIdx.x + k * THREADS;
@@ -246,7 +255,7 @@ rowstep_tall_pass2_kernel(PtrTables t, int first, int rows, int cols, StepScalar
 }
 
 // --------------------------------------------------------------- launchers
-template <typename IO, int VPT, int CLUSTER, int THREADS = kRowThreads>
+template <typename IO, int VPT, int CLUSTER, int THREADS = kRowThreads, bool PREP = true, int MINB = 1>
 static cudaError_t launch_wide_inst(const PtrTables& t, const Group& g, const StepScalars& s,
                                     cudaStream_t stream) {
   const int64_t nrows = (int64_t)g.count * g.rows;
@@ -261,7 +270,7 @@ static cudaError_t launch_wide_inst(const PtrTables& t, const Group& g, const St
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, rowstep_wide_kernel<IO, VPT, CLUSTER, THREADS>, t, g.first, (int)g.rows,
+  return cudaLaunchKernelEx(&cfg, rowstep_wide_kernel<IO, VPT, CLUSTER, THREADS, PREP, MINB>, t, g.first, (int)g.rows,
                             (int)g.cols, s);
 }
 
@@ -280,12 +289,17 @@ static cudaError_t launch_wide(const PtrTables& t, const Group& g, const StepSca
   // Rows up to 32768 elements stay inside one CTA (wider CTAs for longer
   // rows): measured faster than splitting a row over a cluster, whose two
   // cluster barriers cost more than the lower occupancy.
-  if (cols <= 2048) return launch_wide_inst<IO, 1, 1>(t, g, s, stream);
-  if (cols <= 4096) return launch_wide_inst<IO, 2, 1>(t, g, s, stream);
-  if (cols <= 8192) return launch_wide_inst<IO, 2, 1, 512>(t, g, s, stream);
-  if (cols <= 16384) return launch_wide_inst<IO, 4, 1, 512>(t, g, s, stream);
-  if (cols <= 24576) return launch_wide_inst<IO, 3, 1, 1024>(t, g, s, stream);
-  if (cols <= 32768) return launch_wide_inst<IO, 4, 2, 512>(t, g, s, stream);
+  // Rows up to 24576 elements stay inside one CTA; the template arguments are
+  // <IO, vectors per thread, cluster, threads, prefetch W, min CTAs per SM>.
+  // Measured on B200: two or more resident CTAs per SM matter more than
+  // prefetching the parameters before the reduction, and a row split over a
+  // cluster pays two cluster barriers.
+  if (cols <= 2048) return launch_wide_inst<IO, 1, 1, 256, false, 4>(t, g, s, stream);
+  if (cols <= 4096) return launch_wide_inst<IO, 2, 1, 256, false, 4>(t, g, s, stream);
+  if (cols <= 8192) return launch_wide_inst<IO, 2, 1, 512, false, 2>(t, g, s, stream);
+  if (cols <= 16384) return launch_wide_inst<IO, 4, 1, 512, false, 2>(t, g, s, stream);
+  if (cols <= 24576) return launch_wide_inst<IO, 3, 1, 1024, false, 1>(t, g, s, stream);
+  if (cols <= 32768) return launch_wide_inst<IO, 4, 2, 512, false, 1>(t, g, s, stream);
   return launch_wide_inst<IO, 4, 8>(t, g, s, stream);
 }
 

@@ -131,6 +131,17 @@ PRM_API int prm_plan(const prm_ctx* ctx, int64_t step_idx, int* is_refresh,
  * call; the word is cleared. */
 PRM_API int prm_status(prm_ctx* ctx);
 
+/*
+ * Self-test of the device-side failure path.  Every wait inside the kernels
+ * (on TMA, tensor-core and epilogue barriers) is bounded; a wait that runs out
+ * raises the status word and the kernel drains and returns, so the context
+ * stays usable.  This call launches a one-thread kernel that waits limit_ms
+ * (at most 1000) on a barrier nothing completes and then does exactly that:
+ * after it, prm_status returns PRM_ERR_DEVICE_TIMEOUT once and PRM_OK again
+ * afterwards.  Nothing faults, traps or hangs.
+ */
+PRM_API int prm_selftest_timeout(prm_ctx* ctx, double limit_ms, void* cuda_stream);
+
 /* Text of the last error on this handle ("" if none).  Valid until the next
  * call on the handle.  With ctx == NULL: the last prm_create error. */
 PRM_API const char* prm_last_error(const prm_ctx* ctx);

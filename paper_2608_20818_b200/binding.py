@@ -39,7 +39,7 @@ PRM_OPT_NS_WORKSPACE_BYTES = 9
 EXPORTS = (
     "prm_create", "prm_set_option", "prm_workspace_bytes", "prm_set_workspace", "prm_step",
     "prm_step_h2d", "prm_plan", "prm_status", "prm_last_error", "prm_launch_count", "prm_destroy",
-    "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc",
+    "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc", "prm_selftest_timeout",
 )
 PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
 PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_COUNT = 4, 5, 6, 7
@@ -95,6 +95,8 @@ def lib():
                                            c_int, c_float, c_float, c_float, c_float, c_float, c_void_p,
                                            c_char_p, c_size_t]
     L.prm_rowstep_tall_noalloc.restype = c_int
+    L.prm_selftest_timeout.argtypes = [c_void_p, c_double, c_void_p]
+    L.prm_selftest_timeout.restype = c_int
     _lib_handle = L
     return L
 
@@ -189,6 +191,10 @@ def prm_rowstep_tall_noalloc(param, grad, momentum, *, beta, nesterov, lr, wd, g
             float(gamma), float(eps_row), float(scale), c_void_p(s), buf, 256)
     if code != PRM_OK:
         raise PrmError(code, buf.value.decode())
+
+
+def prm_selftest_timeout(h, limit_ms, stream=0):
+    _check(lib().prm_selftest_timeout(h, float(limit_ms), c_void_p(stream)), h)
 
 
 def prm_destroy(h):

@@ -431,6 +431,17 @@ extern "C" int prm_profile_read(prm_ctx* c, double* ms, int64_t* launches, int n
   return dropped ? fail(c, PRM_ERR_STATE, "prm_profile_read: event pool overflowed, totals incomplete") : PRM_OK;
 }
 
+extern "C" int prm_selftest_timeout(prm_ctx* c, double limit_ms, void* cuda_stream) {
+  if (!c) return PRM_ERR_ARG;
+  if (!c->ws) return fail(c, PRM_ERR_WORKSPACE, "prm_selftest_timeout: no workspace attached");
+  if (!(limit_ms > 0) || limit_ms > 1000.0) return fail(c, PRM_ERR_ARG, "prm_selftest_timeout: limit must be in (0, 1000] ms");
+  cudaError_t ce = launch_wait_probe((int*)(c->ws + c->off_status), (uint64_t)(limit_ms * 1e6), nullptr,
+                                     (cudaStream_t)cuda_stream);
+  c->launches += 1;
+  if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("prm_selftest_timeout: ") + cudaGetErrorString(ce));
+  return PRM_OK;
+}
+
 extern "C" const char* prm_last_error(const prm_ctx* c) { return c ? c->err.c_str() : g_create_err.c_str(); }
 
 extern "C" int64_t prm_launch_count(const prm_ctx* c) { return c ? c->launches : 0; }

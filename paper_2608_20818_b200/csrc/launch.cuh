@@ -70,6 +70,9 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
                            cudaStream_t stream, int64_t* launches);
 bool tc_encode_param_map(TcContext* tc, const void* base, int64_t rows, int64_t cols, int tall, void* out128);
 TcContext* tc_create(std::string* err);
+// One thread waits limit_ns on a barrier that never completes, then raises
+// the status word (bit kStatusTimeout) and sets *gave_up (device int, may be null).
+cudaError_t launch_wait_probe(int* status, uint64_t limit_ns, int* gave_up, cudaStream_t stream);
 void tc_destroy(TcContext* tc);
 
 }  // namespace prm

@@ -98,13 +98,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Bounded wait.  Returns false if the CTA is aborting (this or another role
 // ran out of time); the first to give up raises the device status word.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status) {
+                                          int* status, uint64_t limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const uint64_t t0 = global_ns();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > kWaitLimitNs) {
+    if (global_ns() - t0 > limit_ns) {
       *abort_flag = 1;
       atomicOr(status, kStatusTimeout);
       return false;
@@ -543,6 +543,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
   }
 }
 
+// Exercises the bounded wait: one thread waits on a barrier that nothing ever
+// completes, gives up after limit_ns, raises the status word and returns.
+__global__ void wait_probe_kernel(int* status, uint64_t limit_ns, int* gave_up) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const bool ok = mbar_wait(&bar, 0, &abort_flag, status, limit_ns);
+    if (gave_up) *gave_up = ok ? 0 : 1;
+  }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -629,6 +643,11 @@ static bool get_map(TcContext* tc, const void* base, int64_t rows, int64_t kdim,
   if (tc->cache.size() > 4096) tc->cache.clear();
   tc->cache[key] = *out;
   return true;
+}
+
+cudaError_t launch_wait_probe(int* status, uint64_t limit_ns, int* gave_up, cudaStream_t stream) {
+  wait_probe_kernel<<<1, 32, 0, stream>>>(status, limit_ns, gave_up);
+  return cudaGetLastError();
 }
 
 // Tensor map over one bf16 parameter matrix (rows x cols, row-major) for the

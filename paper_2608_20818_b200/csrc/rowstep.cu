@@ -51,7 +51,7 @@ rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
   float acc = 0.f;
 #pragma unroll
   for (int k = 0; k < VPT; ++k) {
-    const int v = v_begin + threadIdx.x + k * THREADS;
+    const int v = v_begin + threadIdx.x + k * (int)blockDim.x;
     if (v < v_end) {
       float gv[8], mv[8];
       load8_stream(g + 8 * v, gv);
@@ -73,7 +73,7 @@ rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
   __syncthreads();
   float total = 0.f;
 #pragma unroll
-  for (int w = 0; w < THREADS / 32; ++w) total += warp_part[w];
+  for (int w = 0; w < THREADS / 32; ++w) total += (w < (int)(blockDim.x >> 5)) ? warp_part[w] : 0.f;
   if constexpr (CLUSTER > 1) {
     cg::cluster_group cluster = cg::this_cluster();
     if (threadIdx.x == 0) cta_part = total;
@@ -88,13 +88,13 @@ rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
   if (!PREP) {
 #pragma unroll
     for (int k = 0; k < VPT; ++k) {
-      const int v = v_begin + threadIdx.x + k * THREADS;
+      const int v = v_begin + threadIdx.x + k * (int)blockDim.x;
       if (v < v_end) pv[k].load_stream(p + 8 * v);
     }
   }
 #pragma unroll
   for (int k = 0; k < VPT; ++k) {
-    const int v = v_begin + threadIdx.x + k * THREADS;
+    const int v = v_begin + threadIdx.x + k * (int)blockDim.x;
     if (v < v_end) {
       float pf[8];
       pv[k].get(pf);
@@ -261,7 +261,12 @@ static cudaError_t launch_wide_inst(const PtrTables& t, const Group& g, const St
   const int64_t nrows = (int64_t)g.count * g.rows;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(nrows * CLUSTER), 1, 1);
-  cfg.blockDim = dim3(THREADS, 1, 1);
+  // Only as many threads as the row needs (whole warps): idle threads would
+  // hold registers and lower the number of resident CTAs.
+  const int part = (int)(((g.cols >> 3) + CLUSTER - 1) / CLUSTER);
+  const int vpt = (part + THREADS - 1) / THREADS;          // vectors per thread actually used (<= VPT)
+  const int need = ((part + vpt - 1) / vpt + 31) / 32 * 32;
+  cfg.blockDim = dim3(need < THREADS ? need : THREADS, 1, 1);
   cfg.stream = stream;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -289,7 +294,7 @@ static cudaError_t launch_wide(const PtrTables& t, const Group& g, const StepSca
   // Rows up to 32768 elements stay inside one CTA (wider CTAs for longer
   // rows): measured faster than splitting a row over a cluster, whose two
   // cluster barriers cost more than the lower occupancy.
-  // Rows up to 24576 elements stay inside one CTA; the template arguments are
+  // Rows up to 32768 elements stay inside one CTA; the template arguments are
   // <IO, vectors per thread, cluster, threads, prefetch W, min CTAs per SM>.
   // Measured on B200: two or more resident CTAs per SM matter more than
   // prefetching the parameters before the reduction, and a row split over a
@@ -299,7 +304,7 @@ static cudaError_t launch_wide(const PtrTables& t, const Group& g, const StepSca
   if (cols <= 8192) return launch_wide_inst<IO, 2, 1, 512, false, 2>(t, g, s, stream);
   if (cols <= 16384) return launch_wide_inst<IO, 4, 1, 512, false, 2>(t, g, s, stream);
   if (cols <= 24576) return launch_wide_inst<IO, 3, 1, 1024, false, 1>(t, g, s, stream);
-  if (cols <= 32768) return launch_wide_inst<IO, 4, 2, 512, false, 1>(t, g, s, stream);
+  if (cols <= 32768) return launch_wide_inst<IO, 4, 1, 1024, false, 1>(t, g, s, stream);
   return launch_wide_inst<IO, 4, 8>(t, g, s, stream);
 }
 

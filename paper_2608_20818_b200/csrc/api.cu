@@ -102,7 +102,7 @@ static void compute_layout(prm_ctx* c) {
       g.tall_scratch_off = off; off = align_up(off + (size_t)g.count * nblk * g.cols * 4, 256);
       g.tall_nu_off = off;      off = align_up(off + (size_t)g.count * g.cols * 4, 256);
     }
-    const size_t per_mat = e * (size_t)(4 * g.rp * g.cp + 2 * g.rp * g.rp);
+    const size_t per_mat = e * (size_t)(2 * g.rp * g.cp + 2 * g.rp * g.rp);   // X ping-pong, A, B
     int nb = (int)std::min<size_t>((size_t)g.count, std::max<size_t>(1, c->ns_budget / per_mat));
     g.ns_batch = nb;
     ns_max = std::max(ns_max, per_mat * nb);
@@ -235,15 +235,14 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
     const int nb = std::min(g.ns_batch, g.count - done);
     char* base = c->ws + c->off_ns;
     char* X[2] = {base, base + e * rc * nb};
-    char* XT[2] = {base + 2 * e * rc * nb, base + 3 * e * rc * nb};
-    char* A = base + 4 * e * rc * nb;
+    char* A = base + 2 * e * rc * nb;
     char* B = A + e * rr * nb;
     const int first = g.first + done;
     cudaError_t ce;
     {
       ProfScope ps(c, PRM_PROF_PREPASS, stream);
-      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, c->check_mode, X[0], XT[0], fro, alpha,
-                             stream, &c->launches);
+      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, c->check_mode, X[0], fro, alpha, stream,
+                             &c->launches);
     }
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("pre-pass: ") + cudaGetErrorString(ce));
     auto gemm = [&](const GemmProblem& pb, const Epilogue& ep, int cls) -> cudaError_t {
@@ -274,14 +273,14 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
       // X <- a X + B X (times alpha in the first iteration); last iteration
       // goes straight into the parameters.
       GemmProblem pu;
-      pu.P = B; pu.Q = XT[cur]; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
+      // (B X)[i,j] = sum_k B[i,k] X[k,j]: X itself is the second operand, read with j contiguous.
+      pu.P = B; pu.Q = X[cur]; pu.q_mn = 1; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
       pu.bs_P = rr; pu.bs_Q = rc; pu.batch = nb; pu.symmetric = 0;
       Epilogue eu;
       eu.k_acc = 1.f; eu.k_aux = kNsA; eu.aux = X[cur]; eu.ld_aux = g.cp; eu.bs_aux = rc;
       if (it == 0) { eu.alpha = alpha; eu.alpha_pow = 1; }
       if (it + 1 < kNsIters) {
         eu.dst = X[cur ^ 1]; eu.ld_dst = g.cp; eu.bs_dst = rc;
-        eu.dst_t = XT[cur ^ 1]; eu.ld_dst_t = g.rp; eu.bs_dst_t = rc;
       } else {
         eu.kind = 1; eu.tables = t; eu.first = first;
         eu.rows = (int)g.rows; eu.cols = (int)g.cols; eu.tall = g.tall ? 1 : 0;

@@ -46,17 +46,19 @@ struct GemmProblem {
   int64_t bs_P = 0, bs_Q = 0;     // batch strides in elements
   int batch = 1;
   int symmetric = 0;
+  int q_mn = 0;                   // Q is stored [batch][Kp][Np] (n contiguous) instead of [batch][Np][Kp]
 };
 
 cudaError_t launch_rowstep(const PtrTables& t, const Group& g, const StepScalars& s, int io_fp32,
                            float* tall_partial, float* tall_nu, cudaStream_t stream,
                            int64_t* launches);
 
-// Momentum update + direction input written to the NS5 workspace in both
-// orientations, with per-CTA partial sums of squares, then alpha per matrix.
-// x_fp32: workspace element type (1: fp32 check mode, 0: bf16).
+// Momentum update + direction input written to the NS5 workspace as the
+// oriented matrix X (r_p x c_p, zero padded), with per-CTA partial sums of
+// squares, then alpha per matrix.  x_fp32: workspace element type (1: fp32
+// check mode, 0: bf16).
 cudaError_t launch_ns_prepass(const PtrTables& t, const Group& g, int first, int batch,
-                              const StepScalars& s, int io_fp32, int x_fp32, void* X, void* XT,
+                              const StepScalars& s, int io_fp32, int x_fp32, void* X,
                               float* fro_partial, float* alpha, cudaStream_t stream,
                               int64_t* launches);
 

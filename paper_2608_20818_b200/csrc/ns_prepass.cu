@@ -2,12 +2,12 @@
 //
 // For every matrix of a sub-batch it updates the momentum in place
 // (Algorithm 1 line 2), forms the direction input U, and writes U - unscaled -
-// into the NS5 workspace in both orientations: X (r x c, the oriented matrix
-// of Section 3.1) and XT (c x r).  All NS5 products then read both operands
-// with the contraction index contiguous.  The Frobenius norm of U is reduced
-// alongside (per-CTA partials, then one fixed-order sum per matrix) and
-// enters the recurrence as alpha = 1/(||U||_F + eps_ns) in the first
-// iteration's epilogues, so the normalisation costs no extra pass.
+// into the NS5 workspace as the oriented matrix X (r x c) of Section 3.1: as
+// stored for wide matrices, transposed through a shared-memory tile for tall
+// ones.  The Frobenius norm of U is reduced alongside (per-CTA partials, then
+// one fixed-order sum per matrix) and enters the recurrence as
+// alpha = 1/(||U||_F + eps_ns) in the first iteration's epilogues, so the
+// normalisation costs no extra pass.
 //
 // The workspace copies are zero-padded to multiples of kPad; zero rows and
 // columns stay zero under X -> aX + (bA + cA^2)X.
@@ -29,8 +29,8 @@ ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
   const int b = blockIdx.z;
   const IO* __restrict__ g = reinterpret_cast<const IO*>(t.grads[first + b]);
   float* __restrict__ m = t.momentum[first + b];
-  XT_* __restrict__ ds = straight + (int64_t)b * bs_s;
-  XT_* __restrict__ dt = transposed + (int64_t)b * bs_t;
+  XT_* __restrict__ ds = straight ? straight + (int64_t)b * bs_s : nullptr;
+  XT_* __restrict__ dt = transposed ? transposed + (int64_t)b * bs_t : nullptr;
   const int r0 = blockIdx.y * kPreTile, c0 = blockIdx.x * kPreTile;
   const int tx = threadIdx.x & 7, ty = threadIdx.x >> 3;   // 8 column vectors x 32 rows
   float acc = 0.f;
@@ -73,7 +73,7 @@ ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
       acc += u[e] * u[e];
       tile[lr][tx * 8 + e] = u[e];
     }
-    store8(ds + (int64_t)row * ld_s + col, u);   // padded extent: always in range
+    if (straight != nullptr) store8(ds + (int64_t)row * ld_s + col, u);   // padded extent: always in range
   }
   acc = warp_sum(acc);
   if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
@@ -84,6 +84,7 @@ ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
     for (int w = 0; w < kPreThreads / 32; ++w) tot += warp_part[w];
     fro_partial[((int64_t)b * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x] = tot;
   }
+  if (transposed == nullptr) return;
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
     const int lc = ty + 32 * half;            // column of the tile = row of the transposed copy
@@ -114,12 +115,12 @@ ns_alpha_kernel(const float* __restrict__ fro_partial, int nparts, float eps_ns,
 
 template <typename IO, typename XT_>
 static cudaError_t prepass_inst(const PtrTables& t, const Group& g, int first, int batch,
-                                const StepScalars& s, XT_* X, XT_* XT, float* fro_partial,
-                                float* alpha, cudaStream_t stream) {
+                                const StepScalars& s, XT_* X, float* fro_partial, float* alpha,
+                                cudaStream_t stream) {
   // Stored extent padded: wide -> (rp, cp), tall -> (cp, rp).
   const int64_t prow = g.tall ? g.cp : g.rp, pcol = g.tall ? g.rp : g.cp;
-  XT_* straight = g.tall ? XT : X;
-  XT_* transposed = g.tall ? X : XT;
+  XT_* straight = g.tall ? nullptr : X;
+  XT_* transposed = g.tall ? X : nullptr;
   const int64_t bs = g.rp * g.cp;
   dim3 grid((unsigned)(pcol / kPreTile), (unsigned)(prow / kPreTile), (unsigned)batch);
   if (grid.y > 65535 || grid.z > 65535) return cudaErrorInvalidValue;
@@ -135,16 +136,16 @@ static cudaError_t prepass_inst(const PtrTables& t, const Group& g, int first, i
 }
 
 cudaError_t launch_ns_prepass(const PtrTables& t, const Group& g, int first, int batch,
-                              const StepScalars& s, int io_fp32, int x_fp32, void* X, void* XT,
+                              const StepScalars& s, int io_fp32, int x_fp32, void* X,
                               float* fro_partial, float* alpha, cudaStream_t stream,
                               int64_t* launches) {
   *launches += 2;
   if (io_fp32) {
-    if (x_fp32) return prepass_inst<float, float>(t, g, first, batch, s, (float*)X, (float*)XT, fro_partial, alpha, stream);
-    return prepass_inst<float, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, (__nv_bfloat16*)XT, fro_partial, alpha, stream);
+    if (x_fp32) return prepass_inst<float, float>(t, g, first, batch, s, (float*)X, fro_partial, alpha, stream);
+    return prepass_inst<float, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, fro_partial, alpha, stream);
   }
-  if (x_fp32) return prepass_inst<__nv_bfloat16, float>(t, g, first, batch, s, (float*)X, (float*)XT, fro_partial, alpha, stream);
-  return prepass_inst<__nv_bfloat16, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, (__nv_bfloat16*)XT, fro_partial, alpha, stream);
+  if (x_fp32) return prepass_inst<__nv_bfloat16, float>(t, g, first, batch, s, (float*)X, fro_partial, alpha, stream);
+  return prepass_inst<__nv_bfloat16, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, fro_partial, alpha, stream);
 }
 
 }  // namespace prm

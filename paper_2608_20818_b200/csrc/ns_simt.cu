@@ -27,8 +27,10 @@ gemm_simt_kernel(GemmProblem pb, Epilogue ep) {
   }
   const float* __restrict__ P = reinterpret_cast<const float*>(pb.P) + (int64_t)b * pb.bs_P +
                                 (int64_t)ti * kSimtTile * pb.Kp;
+  // Q is [Np][Kp] (k contiguous) or, with q_mn, [Kp][Np] (n contiguous).
   const float* __restrict__ Q = reinterpret_cast<const float*>(pb.Q) + (int64_t)b * pb.bs_Q +
-                                (int64_t)tj * kSimtTile * pb.Kp;
+                                (pb.q_mn ? (int64_t)tj * kSimtTile : (int64_t)tj * kSimtTile * pb.Kp);
+  const int qk = threadIdx.x >> 5, qj = (threadIdx.x & 31) * 4;   // q_mn: one float4 of row k per thread
   const int lrow = threadIdx.x >> 1, lk = (threadIdx.x & 1) * 4;
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   float acc[8][8], tot[8][8];
@@ -39,14 +41,20 @@ gemm_simt_kernel(GemmProblem pb, Epilogue ep) {
 
   const int ksteps = (int)(pb.Kp / kSimtK);
   float4 pa = *reinterpret_cast<const float4*>(P + (int64_t)lrow * pb.Kp + lk);
-  float4 qa = *reinterpret_cast<const float4*>(Q + (int64_t)lrow * pb.Kp + lk);
+  float4 qa = pb.q_mn ? *reinterpret_cast<const float4*>(Q + (int64_t)qk * pb.Np + qj)
+                      : *reinterpret_cast<const float4*>(Q + (int64_t)lrow * pb.Kp + lk);
   for (int ks = 0; ks < ksteps; ++ks) {
     As[lk + 0][lrow] = pa.x; As[lk + 1][lrow] = pa.y; As[lk + 2][lrow] = pa.z; As[lk + 3][lrow] = pa.w;
-    Bs[lk + 0][lrow] = qa.x; Bs[lk + 1][lrow] = qa.y; Bs[lk + 2][lrow] = qa.z; Bs[lk + 3][lrow] = qa.w;
+    if (pb.q_mn) {
+      *reinterpret_cast<float4*>(&Bs[qk][qj]) = qa;
+    } else {
+      Bs[lk + 0][lrow] = qa.x; Bs[lk + 1][lrow] = qa.y; Bs[lk + 2][lrow] = qa.z; Bs[lk + 3][lrow] = qa.w;
+    }
     __syncthreads();
     if (ks + 1 < ksteps) {
       pa = *reinterpret_cast<const float4*>(P + (int64_t)lrow * pb.Kp + (ks + 1) * kSimtK + lk);
-      qa = *reinterpret_cast<const float4*>(Q + (int64_t)lrow * pb.Kp + (ks + 1) * kSimtK + lk);
+      qa = pb.q_mn ? *reinterpret_cast<const float4*>(Q + (int64_t)((ks + 1) * kSimtK + qk) * pb.Np + qj)
+                   : *reinterpret_cast<const float4*>(Q + (int64_t)lrow * pb.Kp + (ks + 1) * kSimtK + lk);
     }
 #pragma unroll
     for (int k = 0; k < kSimtK; ++k) {

@@ -174,12 +174,21 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t smem_addr) {
   return (uint64_t)((smem_addr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) |
          (1ull << 46) | (2ull << 61);
 }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+__device__ __forceinline__ uint64_t make_desc_mn(uint32_t smem_addr) {
+  // N-major ("MN-major") operand tile, 128-byte swizzle: each row of 128 bytes
+  // holds 64 consecutive n for one k; 8 such k-rows form a 1024-byte atom.
+  // Atoms follow each other along k every 1024 bytes (stride byte offset) and
+  // along n every 8192 bytes (leading byte offset: the next 64x64 TMA box).
+  return (uint64_t)((smem_addr >> 4) & 0x3FFF) | ((uint64_t)(8192 >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 // Arrives on the barrier at this offset in both CTAs of the pair once all MMAs
@@ -234,7 +243,9 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ,
                const __grid_constant__ CUtensorMap mapAux, const __grid_constant__ CUtensorMap mapDst,
                const __grid_constant__ CUtensorMap mapDstT, int ktiles, int tiles_per_mat,
-               int total_tiles, int symmetric, int mt, Epilogue ep, int* status) {
+               int total_tiles, int symmetric, int mt, int q_mn, Epilogue ep, int* status) {
+  // q_mn: Q is stored [k][n] (n contiguous) instead of [n][k]; its tiles are
+  // loaded as 64x64 boxes and consumed as an N-major MMA operand.
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* ebuf = smem + (size_t)kStages * kStageBytes;           // [kEpiBufs][kEpiBufBytes]
@@ -294,7 +305,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           if (rank == 0) mbar_expect_tx(&full[s], 2 * kStageBytes);
           const uint32_t lead_full = map_to_rank(&full[s], 0);
           tma_load_3d_pair(sa, &mapP, lead_full, kt * kBK, c.ti * kBM, c.b);
-          tma_load_3d_pair(sa + kBytesA, &mapQ, lead_full, kt * kBK, c.tj * kBN + (int)rank * (kBN / 2), c.b);
+          const int n0 = c.tj * kBN + (int)rank * (kBN / 2);      // this CTA's 128 rows (columns) of Q
+          if (!q_mn) {
+            tma_load_3d_pair(sa + kBytesA, &mapQ, lead_full, kt * kBK, n0, c.b);
+          } else {
+            tma_load_3d_pair(sa + kBytesA, &mapQ, lead_full, n0, kt * kBK, c.b);
+            tma_load_3d_pair(sa + kBytesA + kBytesB / 2, &mapQ, lead_full, n0 + 64, kt * kBK, c.b);
+          }
         }
       }
       // Drain: every load issued must have landed before shared memory is
@@ -327,11 +344,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           if (!mbar_wait(&full[s], ph, abort_flag, status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
-          const uint64_t da = make_desc(sa), db = make_desc(sa + kBytesA);
+          const uint64_t da = make_desc(sa);
+          if (!q_mn) {
+            const uint64_t db = make_desc(sa + kBytesA);
 #pragma unroll
-          for (int k = 0; k < kBK / kUmmaK; ++k) {
-            // advance 16 elements = 32 bytes inside the swizzled row: +2 in 16-byte units
-            umma_bf16(tacc, da + 2 * k, db + 2 * k, (kt | k) != 0);
+            for (int k = 0; k < kBK / kUmmaK; ++k) {
+              // advance 16 elements = 32 bytes inside the swizzled row: +2 in 16-byte units
+              umma_bf16(tacc, da + 2 * k, db + 2 * k, kIdesc, (kt | k) != 0);
+            }
+          } else {
+            const uint64_t db = make_desc_mn(sa + kBytesA);
+#pragma unroll
+            for (int k = 0; k < kBK / kUmmaK; ++k) {
+              // Q: 16 k-rows = two 1024-byte atoms further: +128 in 16-byte units
+              umma_bf16(tacc, da + 2 * k, db + 128 * k, kIdesc | (1u << 16), (kt | k) != 0);
+            }
           }
           umma_commit_pair(&empty[s]);        // frees the stage in both CTAs when these MMAs have read it
         }
@@ -675,7 +702,12 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   if (pb.Mp % kBN != 0 || pb.Np % kBN != 0 || pb.Kp % kBK != 0) return cudaErrorInvalidValue;
   CUtensorMap mp, mq, maux, mdst, mdt;
   if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
-  if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
+  if (!pb.q_mn) {
+    if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
+  } else {
+    // Q stored [batch][Kp][Np]: boxes of 64 k-rows x 64 n
+    if (pb.symmetric || !get_map(tc, pb.Q, pb.Kp, pb.Np, pb.batch, 64, &mq)) return cudaErrorInvalidValue;
+  }
   // Epilogue maps (product epilogues only): auxiliary and result slabs of 128
   // rows x 64 columns, transposed result in boxes of 64 x 64.
   maux = mp; mdst = mp; mdt = mp;
@@ -717,7 +749,7 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, gemm_tc_kernel, mp, mq, maux, mdst, mdt, (int)(pb.Kp / kBK), (int)per_mat,
-                            (int)total, pb.symmetric, (int)mt, ep, status);
+                            (int)total, pb.symmetric, (int)mt, pb.q_mn, ep, status);
 }
 
 }  // namespace prm

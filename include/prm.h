@@ -65,6 +65,12 @@ extern "C" {
 #define PRM_OPT_NS_WORKSPACE_BYTES 9 /* soft cap on the NS5 part of the workspace, default
                                    8 GiB; matrices of one shape group are refreshed in
                                    sub-batches that fit.  Before set_workspace. */
+/* Variants of the ablation table (Table 3a of the paper); may be changed between steps. */
+#define PRM_OPT_GAMMA_NS    10  /* multiplier on the NS5 branch, default 1 (the paper's method);
+                                   "scalar-controlled" sets it to gamma */
+#define PRM_OPT_NO_REFRESH  11  /* 1: RowNorm at every step, no NS5 schedule; default 0 */
+
+
 
 typedef struct prm_ctx prm_ctx;
 

@@ -62,6 +62,9 @@ class OracleConfig:
     eps_row: float = 1e-8     # epsilon of Eq. (rownorm)
     eps_ns: float = 1e-7      # epsilon of the NS5 input normalisation
     scale_mode: int = 1       # see shape_scale()
+    # Ablation variants of the paper's Table 3(a):
+    gamma_ns: float = 1.0     # multiplier on the NS5 branch ("scalar-controlled" sets it to gamma)
+    no_refresh: bool = False  # RowNorm at every step (no NS5 schedule)
 
 
 def is_refresh(t: int, K: int) -> bool:
@@ -177,7 +180,7 @@ def direction(U, refresh, cfg: OracleConfig):
     m, n = U.shape
     U_tilde = orient(U)
     if refresh:
-        D_tilde = ns5(U_tilde, cfg.eps_ns)
+        D_tilde = cfg.gamma_ns * ns5(U_tilde, cfg.eps_ns)
     else:
         D_tilde = cfg.gamma * rownorm(U_tilde, cfg.eps_row)
     return orient_inv(D_tilde, m, n)
@@ -194,7 +197,7 @@ def step_matrix(W, G, M_prev, t, cfg: OracleConfig):
     m, n = W.shape
     M_t = momentum_update(M_prev, G, cfg.beta)                 # line 2
     U = direction_input(M_t, G, cfg.beta, cfg.nesterov)
-    refresh = is_refresh(t, cfg.K)                              # line 3
+    refresh = is_refresh(t, cfg.K) and not cfg.no_refresh       # line 3
     D = shape_scale(m, n, cfg.scale_mode) * direction(U, refresh, cfg)  # lines 5-8
     W_next = (1.0 - cfg.lr * cfg.wd) * W - cfg.lr * D           # line 9
     return W_next, M_t

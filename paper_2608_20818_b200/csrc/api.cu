@@ -23,6 +23,8 @@ struct prm_ctx {
   int io_fp32 = 0;
   int check_mode = 0;
   size_t ns_budget = (size_t)8 << 30;
+  float gamma_ns = 1.f;   // multiplier on the NS5 branch (ablation: "scalar-controlled" uses gamma)
+  int no_refresh = 0;     // ablation: RowNorm at every step
 
   std::vector<Group> groups;
   std::vector<int> group_of_mat, order_in_group, slot_of_mat;   // slot = index in pointer tables
@@ -177,6 +179,10 @@ extern "C" int prm_set_option(prm_ctx* c, int key, double v) {
       c->scale_mode = (int)v; return PRM_OK;
     case PRM_OPT_LR: c->lr = (float)v; return PRM_OK;
     case PRM_OPT_WD: c->wd = (float)v; return PRM_OK;
+    case PRM_OPT_GAMMA_NS: if (!(v > 0)) return fail(c, PRM_ERR_ARG, "gamma_ns must be > 0"); c->gamma_ns = (float)v; return PRM_OK;
+    case PRM_OPT_NO_REFRESH:
+      if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
+      c->no_refresh = (int)v; return PRM_OK;
     case PRM_OPT_IO_DTYPE:
     case PRM_OPT_CHECK_MODE:
     case PRM_OPT_NS_WORKSPACE_BYTES:
@@ -217,7 +223,7 @@ extern "C" int prm_set_workspace(prm_ctx* c, void* dev_ptr, size_t bytes) {
 extern "C" int prm_plan(const prm_ctx* c, int64_t step_idx, int* is_refresh, int* n_groups,
                         int* group_of_mat, int* order_in_group) {
   if (!c || step_idx < 0) return PRM_ERR_ARG;
-  if (is_refresh) *is_refresh = (step_idx % c->K) == 0 ? 1 : 0;
+  if (is_refresh) *is_refresh = ((step_idx % c->K) == 0 && !c->no_refresh) ? 1 : 0;
   if (n_groups) *n_groups = (int)c->groups.size();
   if (group_of_mat) memcpy(group_of_mat, c->group_of_mat.data(), sizeof(int) * c->n_mats);
   if (order_in_group) memcpy(order_in_group, c->order_in_group.data(), sizeof(int) * c->n_mats);
@@ -284,7 +290,7 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
       } else {
         eu.kind = 1; eu.tables = t; eu.first = first;
         eu.rows = (int)g.rows; eu.cols = (int)g.cols; eu.tall = g.tall ? 1 : 0;
-        eu.io_fp32 = c->io_fp32; eu.decay = s.decay; eu.lr_s = s.lr_s;
+        eu.io_fp32 = c->io_fp32; eu.decay = s.decay; eu.lr_s = s.lr_s * c->gamma_ns;
         // bf16 parameters with 16-byte aligned rows are updated through TMA-staged tiles.
         if (!c->check_mode && !c->io_fp32 && g.cols % 8 == 0) eu.param_maps = c->ws + c->off_pmaps;
       }
@@ -348,7 +354,7 @@ static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
   t.params = tb;
   t.grads = (const void**)(tb + n);
   t.momentum = (float**)(tb + 2 * n);
-  const bool refresh = (step_idx % c->K) == 0;
+  const bool refresh = (step_idx % c->K) == 0 && !c->no_refresh;
   for (const Group& g : c->groups) {
     StepScalars s;
     s.beta = c->beta; s.omb = 1.f - c->beta; s.nesterov = c->nesterov;

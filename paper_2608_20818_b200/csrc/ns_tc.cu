@@ -45,13 +45,13 @@ constexpr int kBM = 128;          // tile rows  (UMMA M)
 constexpr int kBN = 256;          // tile cols  (UMMA N)
 constexpr int kBK = 64;           // k per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
-constexpr int kStages = 5;
+constexpr int kStages = 4;
 constexpr int kEpiWarps = 8;         // two warps per TMEM lane quadrant
 constexpr int kIoWarp = 2 + kEpiWarps;
 constexpr int kTcThreads = 32 * (kIoWarp + 1);
 constexpr int kSlabCols = 64;        // epilogue slab: 128 rows x 64 columns
 constexpr int kSlabs = 4;            // slabs per tile (kBN / kSlabCols)
-constexpr int kEpiBufs = 2;
+constexpr int kEpiBufs = 3;
 constexpr uint32_t kSlabBytes = 128 * kSlabCols * 2;        // result slab, also the aux slab
 constexpr uint32_t kEpiBufBytes = 2 * kSlabBytes;           // + transposed slab (2 boxes of 64x64)
 constexpr uint32_t kBytesA = kBM * kBK * 2;

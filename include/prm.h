@@ -112,10 +112,14 @@ PRM_API int prm_step(prm_ctx* ctx, void* const* params, const void* const* grads
              float* const* momentum, int64_t step_idx, void* cuda_stream);
 
 /*
- * Same step, but first copies this step's gradients from HOST memory:
+ * Same step, but this step's gradients come from HOST memory:
  * grads_host[i] (rows*cols elements of the I/O dtype, ideally pinned) is
- * copied to grads_dev[i] with one asynchronous copy per matrix on the stream,
- * then the step runs as in prm_step.
+ * copied to grads_dev[i] with one asynchronous copy per matrix, then the step
+ * runs as in prm_step.  The copies run on a stream owned by the handle,
+ * ordered after everything already queued on cuda_stream; the kernels of a
+ * shape group wait only for that group's gradients, so the copy of the next
+ * group overlaps the work of the current one.  Everything the call enqueues is
+ * complete when cuda_stream is.
  */
 PRM_API int prm_step_h2d(prm_ctx* ctx, void* const* params, void* const* grads_dev,
                  const void* const* grads_host, float* const* momentum,

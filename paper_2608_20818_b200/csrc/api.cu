@@ -48,6 +48,13 @@ struct prm_ctx {
   std::vector<int64_t> prof_launches;   // kernel launches inside pair i
   size_t prof_used = 0;
   int64_t prof_dropped = 0;
+
+  // prm_step_h2d: gradients travel on a copy stream, one event per shape group,
+  // so the copy of group g+1 overlaps the kernels of group g (host resources,
+  // created on first use)
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t copy_begin = nullptr;
+  std::vector<cudaEvent_t> copy_done;   // per group
 };
 
 namespace {
@@ -342,12 +349,29 @@ static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
   }
   if (grads_host) {
     const size_t esz = c->io_fp32 ? 4 : 2;
-    for (int i = 0; i < n; ++i) {
+    for (int i = 0; i < n; ++i)
       if (!grads_host[i]) return fail(c, PRM_ERR_ARG, "prm_step_h2d: NULL host gradient pointer");
-      ce = cudaMemcpyAsync(grads_dev[i], grads_host[i], esz * (size_t)c->shapes[2 * i] * (size_t)c->shapes[2 * i + 1],
-                           cudaMemcpyHostToDevice, stream);
-      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("gradient copy: ") + cudaGetErrorString(ce));
+    if (!c->copy_stream) {
+      ce = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+      if (ce == cudaSuccess) ce = cudaEventCreateWithFlags(&c->copy_begin, cudaEventDisableTiming);
+      c->copy_done.assign(c->groups.size(), nullptr);
+      for (size_t k = 0; k < c->groups.size() && ce == cudaSuccess; ++k)
+        ce = cudaEventCreateWithFlags(&c->copy_done[k], cudaEventDisableTiming);
+      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("copy stream: ") + cudaGetErrorString(ce));
     }
+    // The copies may not overtake work already queued on the caller's stream
+    // (the previous step still reads the gradient buffers).
+    ce = cudaEventRecord(c->copy_begin, stream);
+    if (ce == cudaSuccess) ce = cudaStreamWaitEvent(c->copy_stream, c->copy_begin, 0);
+    for (size_t k = 0; k < c->groups.size() && ce == cudaSuccess; ++k) {
+      for (int i = 0; i < n && ce == cudaSuccess; ++i) {
+        if (c->group_of_mat[i] != (int)k) continue;
+        ce = cudaMemcpyAsync(grads_dev[i], grads_host[i], esz * (size_t)c->shapes[2 * i] * (size_t)c->shapes[2 * i + 1],
+                             cudaMemcpyHostToDevice, c->copy_stream);
+      }
+      if (ce == cudaSuccess) ce = cudaEventRecord(c->copy_done[k], c->copy_stream);
+    }
+    if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("gradient copy: ") + cudaGetErrorString(ce));
   }
   PtrTables t;
   void** tb = (void**)(c->ws + c->off_tables);
@@ -355,7 +379,12 @@ static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
   t.grads = (const void**)(tb + n);
   t.momentum = (float**)(tb + 2 * n);
   const bool refresh = (step_idx % c->K) == 0 && !c->no_refresh;
-  for (const Group& g : c->groups) {
+  for (size_t gi = 0; gi < c->groups.size(); ++gi) {
+    const Group& g = c->groups[gi];
+    if (grads_host) {
+      ce = cudaStreamWaitEvent(stream, c->copy_done[gi], 0);   // this group's gradients have landed
+      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("gradient copy: ") + cudaGetErrorString(ce));
+    }
     StepScalars s;
     s.beta = c->beta; s.omb = 1.f - c->beta; s.nesterov = c->nesterov;
     s.decay = 1.f - c->lr * c->wd;
@@ -455,6 +484,9 @@ extern "C" int prm_destroy(prm_ctx* c) {
   if (!c) return PRM_ERR_ARG;
   if (c->tc) tc_destroy(c->tc);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->copy_done) if (e) cudaEventDestroy(e);
+  if (c->copy_begin) cudaEventDestroy(c->copy_begin);
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   delete c;
   return PRM_OK;
 }

@@ -216,6 +216,24 @@ PRM_API int prm_rowstep_tall_noalloc(void* param, const void* grad, float* momen
                                      float scale, void* cuda_stream, char* errbuf,
                                      size_t errbuf_len);
 
+/*
+ * AdamW for the parameters outside the Muon set (Algorithm 1 line 11: biases,
+ * normalisation parameters and everything outside the transformer blocks keep
+ * "the same AdamW rule as the baseline"; hyper-parameter table: lr 1e-4,
+ * betas (0.9, 0.95), eps 1e-8, weight decay 0.01).  Decoupled form with bias
+ * correction, step >= 1 is the 1-based step count:
+ *   p <- p*(1 - lr*wd);  m <- beta1*m + (1-beta1)*g;  v <- beta2*v + (1-beta2)*g^2
+ *   p <- p - lr * (m/(1-beta1^step)) / (sqrt(v/(1-beta2^step)) + eps)
+ * params/grads/exp_avg/exp_avg_sq: HOST arrays of n_tensors DEVICE pointers
+ * (16-byte aligned); tensor i holds numel[i] contiguous elements of any shape;
+ * params and grads are bf16 (io_fp32 = 0) or fp32, the moments fp32, all
+ * updated in place.  Needs no handle and no workspace; enqueues on cuda_stream.
+ */
+PRM_API int prm_adamw_step(int n_tensors, void* const* params, const void* const* grads,
+                           float* const* exp_avg, float* const* exp_avg_sq, const int64_t* numel,
+                           int io_fp32, float lr, float beta1, float beta2, float eps, float wd,
+                           int64_t step, void* cuda_stream);
+
 /* Frees host resources.  Device memory belongs to the caller. */
 PRM_API int prm_destroy(prm_ctx* ctx);
 

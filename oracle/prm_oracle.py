@@ -211,3 +211,23 @@ def step(params, grads, momenta, t, cfg: OracleConfig):
         W_out.append(Wn)
         M_out.append(Mn)
     return W_out, M_out
+
+
+def adamw_step(p, g, m, v, t, lr=1e-4, beta1=0.9, beta2=0.95, eps=1e-8, wd=0.01):
+    """One AdamW step for a parameter outside the Muon set (Algorithm 1 line 11:
+    "the same AdamW rule as the baseline"; hyper-parameter table: lr 1e-4,
+    betas (0.9, 0.95), eps 1e-8, weight decay 0.01).  The paper does not spell
+    the rule out; this is the usual decoupled form with bias correction:
+        p <- p*(1 - lr*wd)
+        m <- beta1*m + (1-beta1)*g,   v <- beta2*v + (1-beta2)*g^2
+        p <- p - lr * (m/(1-beta1^t)) / (sqrt(v/(1-beta2^t)) + eps)
+    with t the 1-based step count.  Returns (p, m, v) in fp64."""
+    p = np.asarray(p, dtype=np.float64)
+    g = np.asarray(g, dtype=np.float64)
+    m = beta1 * np.asarray(m, dtype=np.float64) + (1.0 - beta1) * g
+    v = beta2 * np.asarray(v, dtype=np.float64) + (1.0 - beta2) * g * g
+    p = p * (1.0 - lr * wd)
+    m_hat = m / (1.0 - beta1 ** t)
+    v_hat = v / (1.0 - beta2 ** t)
+    p = p - lr * m_hat / (np.sqrt(v_hat) + eps)
+    return p, m, v

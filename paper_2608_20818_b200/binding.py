@@ -41,7 +41,7 @@ PRM_OPT_NO_REFRESH = 11
 EXPORTS = (
     "prm_create", "prm_set_option", "prm_workspace_bytes", "prm_set_workspace", "prm_step",
     "prm_step_h2d", "prm_plan", "prm_status", "prm_last_error", "prm_launch_count", "prm_destroy",
-    "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc", "prm_selftest_timeout",
+    "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc", "prm_selftest_timeout", "prm_adamw_step",
 )
 PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
 PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_COUNT = 4, 5, 6, 7
@@ -99,6 +99,10 @@ def lib():
     L.prm_rowstep_tall_noalloc.restype = c_int
     L.prm_selftest_timeout.argtypes = [c_void_p, c_double, c_void_p]
     L.prm_selftest_timeout.restype = c_int
+    L.prm_adamw_step.argtypes = [c_int, POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p), POINTER(c_void_p),
+                                 POINTER(c_int64), c_int, c_float, c_float, c_float, c_float, c_float, c_int64,
+                                 c_void_p]
+    L.prm_adamw_step.restype = c_int
     _lib_handle = L
     return L
 
@@ -197,6 +201,24 @@ def prm_rowstep_tall_noalloc(param, grad, momentum, *, beta, nesterov, lr, wd, g
 
 def prm_selftest_timeout(h, limit_ms, stream=0):
     _check(lib().prm_selftest_timeout(h, float(limit_ms), c_void_p(stream)), h)
+
+
+def prm_adamw_step(params, grads, exp_avg, exp_avg_sq, step, *, lr=1e-4, beta1=0.9, beta2=0.95, eps=1e-8, wd=0.01,
+                   stream=None):
+    """AdamW on a list of device tensors of any shape (the parameters outside
+    the Muon set), in place; step is the 1-based step count."""
+    n = len(params)
+    if n == 0:
+        return
+    io_fp32 = 1 if params[0].dtype == torch.float32 else 0
+    numel = (c_int64 * n)(*[p.numel() for p in params])
+    s = (stream or torch.cuda.current_stream(params[0].device)).cuda_stream
+    with torch.cuda.device(params[0].device):
+        code = lib().prm_adamw_step(n, _ptr_array(params), _ptr_array(grads), _ptr_array(exp_avg),
+                                    _ptr_array(exp_avg_sq), numel, io_fp32, float(lr), float(beta1), float(beta2),
+                                    float(eps), float(wd), int(step), c_void_p(s))
+    if code != PRM_OK:
+        raise PrmError(code, "prm_adamw_step failed")
 
 
 def prm_destroy(h):

@@ -132,11 +132,14 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------- CPU oracle
-def oracle_sample(wl, K, budget_s=10.0):
-    """Times the fp64 oracle on a bounded sample of the workload and scales it
-    to the whole shape set: one refresh and one row step on a square r x r
-    matrix (r <= d chosen so the refresh fits the time budget), scaled by the
-    paper's flop model (refresh) and by element count (row step)."""
+def oracle_sample(wl, K, budget_s=20.0):
+    """Times the fp64 oracle, as it stands, on a bounded sample of the workload
+    and scales it to the whole shape set.  The sample is one matrix of each of
+    the first distinct shapes of the set, as many as are predicted to fit the
+    time budget (always at least one; a square matrix smaller than d x d when
+    even that does not fit); each gets one refresh and one row step.  The
+    refresh is scaled by the paper's flop model 20r^2c+10r^3, the row step by
+    element count."""
     import numpy as np
     from oracle import prm_oracle as O
     try:
@@ -146,31 +149,46 @@ def oracle_sample(wl, K, budget_s=10.0):
         cores = os.cpu_count() or 1
     cfg = O.OracleConfig(K=K, beta=wl.beta, nesterov=wl.nesterov, lr=wl.lr, wd=wl.wd, gamma=wl.gamma)
     rng = np.random.default_rng(20818)
-    d = max(min(m, n) for (m, n) in wl.shapes)
 
-    def one(r, t):
-        W = rng.standard_normal((r, r)) * 0.02
-        G = rng.standard_normal((r, r)) * wl.grad_std
-        M = rng.standard_normal((r, r)) * wl.grad_std
+    def one(shape, t):
+        W = rng.standard_normal(shape) * 0.02
+        G = rng.standard_normal(shape) * wl.grad_std
+        M = rng.standard_normal(shape) * wl.grad_std
         t0 = time.perf_counter()
         O.step_matrix(W, G, M, t, cfg)
         return time.perf_counter() - t0
 
-    probe = min(d, 512)
+    def model(shape):
+        r, c = min(shape), max(shape)
+        return 20.0 * r * r * c + 10.0 * r ** 3
+
+    distinct = []
+    for sh in wl.shapes:
+        if sh not in distinct:
+            distinct.append(sh)
+    distinct.sort(key=model)
+    probe = (min(512, min(distinct[0])),) * 2
     one(probe, 0)
-    rate = 30.0 * probe ** 3 / max(one(probe, 0), 1e-6)          # flop/s of the refresh at probe size
-    r = int(min(d, max(probe, (budget_s * rate / 30.0) ** (1.0 / 3.0)))) // 64 * 64
-    r = max(r, min(d, 64))
-    t_ref = one(r, 0)
-    t_row = one(r, 1) if K > 1 else 0.0
-    _, model = ns5_flops(wl.shapes)
-    ref_ms = 1e3 * t_ref * model / (30.0 * r ** 3)
-    row_ms = 1e3 * t_row * elements(wl.shapes) / float(r * r)
+    rate = model(probe) / max(one(probe, 0), 1e-6)           # flop/s of the refresh at probe size
+    sample, predicted = [], 0.0
+    for sh in distinct:
+        if sample and predicted + model(sh) / rate > budget_s:
+            break
+        sample.append(sh)
+        predicted += model(sh) / rate
+    if len(sample) == 1 and model(sample[0]) / rate > budget_s:   # shrink the only matrix
+        r = max(64, int((budget_s * rate / 30.0) ** (1.0 / 3.0)) // 64 * 64)
+        sample = [(min(r, min(sample[0])),) * 2]
+    t_ref = sum(one(sh, 0) for sh in sample)
+    t_row = sum(one(sh, 1) for sh in sample) if K > 1 else 0.0
+    _, total_model = ns5_flops(wl.shapes)
+    ref_ms = 1e3 * t_ref * total_model / sum(model(sh) for sh in sample)
+    row_ms = 1e3 * t_row * elements(wl.shapes) / float(sum(m * n for (m, n) in sample))
     amort = (ref_ms + (K - 1) * row_ms) / K
-    sample = (f"one refresh and one row step of the oracle on a {r}x{r} matrix "
-              f"({t_ref:.2f} s, {t_row:.3f} s), scaled to the shape set by the 20r^2c+10r^3 flop model "
-              f"(refresh) and by element count (row step)")
-    return {"value": amort, "unit": "ms/step", "cores": cores, "kind": "oracle", "sample": sample,
+    txt = (f"one refresh and one row step of the oracle on one matrix each of {sample} "
+           f"({t_ref:.2f} s, {t_row:.3f} s), scaled to the shape set by the 20r^2c+10r^3 flop model "
+           f"(refresh) and by element count (row step)")
+    return {"value": amort, "unit": "ms/step", "cores": cores, "kind": "oracle", "sample": txt,
             "refresh_ms": ref_ms, "row_step_ms": row_ms}
 
 
@@ -181,7 +199,7 @@ def run_reference(args, wl, K):
         return
     vals = []
     base = None
-    per = max(2.0, min(10.0, 120.0 / max(1, args.steps + args.warmup)))
+    per = max(2.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
     for i in range(args.warmup + args.steps):
         base = oracle_sample(wl, K, budget_s=per)
         if i >= args.warmup:

@@ -113,7 +113,11 @@ static void compute_layout(prm_ctx* c) {
     }
     const size_t per_mat = e * (size_t)(2 * g.rp * g.cp + 2 * g.rp * g.rp);   // X ping-pong, A, B
     int nb = (int)std::min<size_t>((size_t)g.count, std::max<size_t>(1, c->ns_budget / per_mat));
+    // equal sub-batches: 42 matrices with room for 18 run as 14+14+14, not 18+18+6
+    const int chunks = (g.count + nb - 1) / nb;
+    nb = (g.count + chunks - 1) / chunks;
     g.ns_batch = nb;
+
     ns_max = std::max(ns_max, per_mat * nb);
     fro_max = std::max(fro_max, (size_t)nb * (size_t)((g.rp / 64) * (g.cp / 64)));
     batch_max = std::max(batch_max, nb);

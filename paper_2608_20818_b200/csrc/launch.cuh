@@ -5,12 +5,11 @@
 
 namespace prm {
 
-// Epilogue of every NS5 product D[i,j] = sum_k P[i,k]*Q[j,k] (both operands
-// row-major with k contiguous).  With f = alpha[b]^alpha_pow (1 if alpha is
-// null) and v = f*(k_acc*D[i,j] + k_aux*aux[i,j]):
-//   kind 0: dst[i,j] = v; if dst_t is set, dst_t[j,i] = v as well (for the
-//           symmetric products this is the mirror write of the other
-//           triangle, for the X update it is the transposed copy of X).
+// Epilogue of every NS5 product D[i,j] = sum_k P[i,k]*Q[j,k].  With
+// f = alpha[b]^alpha_pow (1 if alpha is null) and
+// v = f*(k_acc*D[i,j] + k_aux*aux[i,j]):
+//   kind 0: dst[i,j] = v; if dst_t is set, dst_t[j,i] = v as well (the mirror
+//           write of the other triangle of a symmetric product).
 //   kind 1: parameter update W = decay*W - lr_s*v at the stored position of
 //           oriented element (i,j) (Eq. periodic-direction, rho_t = 1).
 struct Epilogue {

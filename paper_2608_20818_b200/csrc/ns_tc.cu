@@ -1,7 +1,8 @@
 // Tensor-core NS5 products for sm_100a: D[i,j] = sum_k P[i,k]*Q[j,k] with bf16
 // operands, fp32 accumulation in tensor memory, and the fused epilogues of
-// struct Epilogue (polynomial coefficients, Frobenius scale, mirror write,
-// transposed copy of X, final parameter update).
+// struct Epilogue (polynomial coefficients, Frobenius scale, mirror write of
+// the symmetric products, final parameter update).  Q may also be stored
+// [k][n] (N-major operand), which is how the update product reads X.
 //
 // Persistent CTA pairs (clusters of two CTAs on two SMs), 352 threads per CTA.
 // A pair computes a 256x256 tile with tcgen05.mma.cta_group::2: each CTA holds

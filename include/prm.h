@@ -234,6 +234,35 @@ PRM_API int prm_adamw_step(int n_tensors, void* const* params, const void* const
                            int io_fp32, float lr, float beta1, float beta2, float eps, float wd,
                            int64_t step, void* cuda_stream);
 
+/*
+ * Sharded tall RowNorm (Section 3.3, Eq. sharded-tall-rownorm; Algorithm 2
+ * lines 9-13): the row step of a tall matrix (global rows > cols) whose rows
+ * are split over ranks.  Each rank holds rows_local consecutive rows.
+ *
+ * prm_tall_shard_stats   updates the local momentum rows in place and writes
+ *   the local column sums of squares of the direction input, colsumsq_out[j] =
+ *   sum over local rows of U_ij^2 (cols floats, device; no square root).
+ *   scratch: device, prm_tall_shard_scratch_bytes(rows_local, cols) bytes.
+ * The caller then SUMS colsumsq over all ranks (one all-reduce of cols floats
+ * per matrix; the buffers of all tall matrices may be packed into one).
+ * prm_tall_shard_apply    finishes the local rows with the global sums:
+ *   nu_j = max(sqrt(colsumsq[j]), eps_row) (square root first, then the clamp),
+ *   W_ij <- (1 - lr*wd) W_ij - lr*scale*gamma*U_ij/nu_j, where scale is s(W) of
+ *   the GLOBAL shape, e.g. sqrt(global_rows/cols).
+ * Both need cols % 8 == 0 and 16-byte aligned pointers; params/grads bf16
+ * (io_fp32 = 0) or fp32, momentum fp32.  With one shard holding all rows the
+ * pair computes exactly prm_step's tall row step.
+ */
+PRM_API size_t prm_tall_shard_scratch_bytes(int64_t rows_local, int64_t cols);
+PRM_API int prm_tall_shard_stats(const void* grad_shard, float* momentum_shard, int64_t rows_local,
+                                 int64_t cols, int io_fp32, float beta, int nesterov,
+                                 float* colsumsq_out, float* scratch, size_t scratch_bytes,
+                                 void* cuda_stream);
+PRM_API int prm_tall_shard_apply(void* param_shard, const void* grad_shard, const float* momentum_shard,
+                                 int64_t rows_local, int64_t cols, int io_fp32, float beta, int nesterov,
+                                 float lr, float wd, float gamma, float eps_row, float scale,
+                                 const float* colsumsq, void* cuda_stream);
+
 /* Frees host resources.  Device memory belongs to the caller. */
 PRM_API int prm_destroy(prm_ctx* ctx);
 

@@ -42,6 +42,7 @@ EXPORTS = (
     "prm_create", "prm_set_option", "prm_workspace_bytes", "prm_set_workspace", "prm_step",
     "prm_step_h2d", "prm_plan", "prm_status", "prm_last_error", "prm_launch_count", "prm_destroy",
     "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc", "prm_selftest_timeout", "prm_adamw_step",
+    "prm_tall_shard_scratch_bytes", "prm_tall_shard_stats", "prm_tall_shard_apply",
 )
 PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
 PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_COUNT = 4, 5, 6, 7
@@ -103,6 +104,14 @@ def lib():
                                  POINTER(c_int64), c_int, c_float, c_float, c_float, c_float, c_float, c_int64,
                                  c_void_p]
     L.prm_adamw_step.restype = c_int
+    L.prm_tall_shard_scratch_bytes.argtypes = [c_int64, c_int64]
+    L.prm_tall_shard_scratch_bytes.restype = c_size_t
+    L.prm_tall_shard_stats.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int, c_float, c_int, c_void_p, c_void_p,
+                                       c_size_t, c_void_p]
+    L.prm_tall_shard_stats.restype = c_int
+    L.prm_tall_shard_apply.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int, c_float, c_int, c_float,
+                                       c_float, c_float, c_float, c_float, c_void_p, c_void_p]
+    L.prm_tall_shard_apply.restype = c_int
     _lib_handle = L
     return L
 

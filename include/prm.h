@@ -188,8 +188,9 @@ PRM_API int prm_profile_read(prm_ctx* ctx, double* ms, int64_t* launches, int n_
  * already owns the GPU's memory, or a loop that must stay clear of the
  * device-wide synchronisation inside cudaMalloc/cudaFree.  The column
  * partial sums and column norms that the tall row step needs live in a fixed
- * 4 MiB array inside the library image (held by every GPU that loads the
- * library, until the process exits).  The call itself performs no cudaMalloc,
+ * 4 MiB array inside the library image (held by every GPU that uses the
+ * library, from the moment the driver loads the module until the process
+ * exits).  The call itself performs no cudaMalloc,
  * cudaFree or other allocating call.
  *
  *   param, grad   device pointers, rows x cols row-major, bf16 (io_fp32 = 0)

@@ -274,24 +274,22 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
       pa.P = X[cur]; pa.Q = X[cur]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
       pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
       Epilogue ea;
-      ea.dst = A; ea.ld_dst = g.rp; ea.bs_dst = rr;
-      ea.dst_t = A; ea.ld_dst_t = g.rp; ea.bs_dst_t = rr;
+      ea.dst = A; ea.ld_dst = g.rp; ea.bs_dst = rr;   // blocks on and below the diagonal only
       if (it == 0) { ea.alpha = alpha; ea.alpha_pow = 2; }
       if ((ce = gemm(pa, ea, PRM_PROF_GRAM)) != cudaSuccess) break;
       // B = b A + c A^2
       GemmProblem pp;
       pp.P = A; pp.Q = A; pp.Mp = g.rp; pp.Np = g.rp; pp.Kp = g.rp;
-      pp.bs_P = rr; pp.bs_Q = rr; pp.batch = nb; pp.symmetric = 1;
+      pp.bs_P = rr; pp.bs_Q = rr; pp.batch = nb; pp.symmetric = 1; pp.sym_ops = 3;
       Epilogue eb;
       eb.k_acc = kNsC; eb.k_aux = kNsB; eb.aux = A; eb.ld_aux = g.rp; eb.bs_aux = rr;
       eb.dst = B; eb.ld_dst = g.rp; eb.bs_dst = rr;
-      eb.dst_t = B; eb.ld_dst_t = g.rp; eb.bs_dst_t = rr;
       if ((ce = gemm(pp, eb, PRM_PROF_POLY)) != cudaSuccess) break;
       // X <- a X + B X (times alpha in the first iteration); last iteration
       // goes straight into the parameters.
       GemmProblem pu;
       // (B X)[i,j] = sum_k B[i,k] X[k,j]: X itself is the second operand, read with j contiguous.
-      pu.P = B; pu.Q = X[cur]; pu.q_mn = 1; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
+      pu.P = B; pu.Q = X[cur]; pu.q_mn = 1; pu.sym_ops = 1; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
       pu.bs_P = rr; pu.bs_Q = rc; pu.batch = nb; pu.symmetric = 0;
       Epilogue eu;
       eu.k_acc = 1.f; eu.k_aux = kNsA; eu.aux = X[cur]; eu.ld_aux = g.cp; eu.bs_aux = rc;

@@ -8,8 +8,10 @@ namespace prm {
 // Epilogue of every NS5 product D[i,j] = sum_k P[i,k]*Q[j,k].  With
 // f = alpha[b]^alpha_pow (1 if alpha is null) and
 // v = f*(k_acc*D[i,j] + k_aux*aux[i,j]):
-//   kind 0: dst[i,j] = v; if dst_t is set, dst_t[j,i] = v as well (the mirror
-//           write of the other triangle of a symmetric product).
+//   kind 0: dst[i,j] = v; if dst_t is set, dst_t[j,i] = v as well.  The
+//           symmetric products store only the blocks they compute (on and
+//           below the diagonal); their consumers read the mirrored block
+//           instead of the missing one (GemmProblem::sym_ops).
 //   kind 1: parameter update W = decay*W - lr_s*v at the stored position of
 //           oriented element (i,j) (Eq. periodic-direction, rho_t = 1).
 struct Epilogue {
@@ -46,6 +48,9 @@ struct GemmProblem {
   int batch = 1;
   int symmetric = 0;
   int q_mn = 0;                   // Q is stored [batch][Kp][Np] (n contiguous) instead of [batch][Np][Kp]
+  // Bit 0: P, bit 1: Q is a symmetric matrix of which only the 256x256 blocks on
+  // and below the diagonal are stored; the rest is read from the mirrored block.
+  int sym_ops = 0;
 };
 
 cudaError_t launch_rowstep(const PtrTables& t, const Group& g, const StepScalars& s, int io_fp32,

@@ -19,19 +19,20 @@ gemm_simt_kernel(GemmProblem pb, Epilogue ep) {
   const int b = blockIdx.y;
   int ti, tj;
   if (pb.symmetric) {
-    tri_decode(blockIdx.x, ti, tj);
+    // every 128x128 tile of the 256x256 blocks on and below the diagonal
+    int bi, bj;
+    tri_decode(blockIdx.x >> 2, bi, bj);
+    ti = 2 * bi + ((blockIdx.x >> 1) & 1);
+    tj = 2 * bj + (blockIdx.x & 1);
   } else {
     const int nt = (int)(pb.Np / kSimtTile);
     ti = blockIdx.x / nt;
     tj = blockIdx.x % nt;
   }
-  const float* __restrict__ P = reinterpret_cast<const float*>(pb.P) + (int64_t)b * pb.bs_P +
-                                (int64_t)ti * kSimtTile * pb.Kp;
-  // Q is [Np][Kp] (k contiguous) or, with q_mn, [Kp][Np] (n contiguous).
-  const float* __restrict__ Q = reinterpret_cast<const float*>(pb.Q) + (int64_t)b * pb.bs_Q +
-                                (pb.q_mn ? (int64_t)tj * kSimtTile : (int64_t)tj * kSimtTile * pb.Kp);
-  const int qk = threadIdx.x >> 5, qj = (threadIdx.x & 31) * 4;   // q_mn: one float4 of row k per thread
-  const int lrow = threadIdx.x >> 1, lk = (threadIdx.x & 1) * 4;
+  const float* __restrict__ P = reinterpret_cast<const float*>(pb.P) + (int64_t)b * pb.bs_P;
+  const float* __restrict__ Q = reinterpret_cast<const float*>(pb.Q) + (int64_t)b * pb.bs_Q;
+  const int qk = threadIdx.x >> 5, qj = (threadIdx.x & 31) * 4;   // transposed storage: one float4 of row k per thread
+  const int lrow = threadIdx.x >> 1, lk = (threadIdx.x & 1) * 4;  // k-contiguous storage: four k of one row per thread
   const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
   float acc[8][8], tot[8][8];
 #pragma unroll
@@ -39,22 +40,37 @@ gemm_simt_kernel(GemmProblem pb, Epilogue ep) {
 #pragma unroll
     for (int c = 0; c < 8; ++c) { acc[a][c] = 0.f; tot[a][c] = 0.f; }
 
+  // Where the 8 x 128 operand slice of k-step ks lives.  A symmetric operand
+  // (sym_ops) is stored only in the 256x256 blocks on and below the diagonal:
+  // right of its diagonal block the slice is read from the mirrored block,
+  // which is stored [k][row].  Q with q_mn is stored [k][n] throughout.
+  auto p_transposed = [&](int ks) { return (pb.sym_ops & 1) && (ks * kSimtK) / kPad > (ti * kSimtTile) / kPad; };
+  auto q_transposed = [&](int ks) {
+    return pb.q_mn || ((pb.sym_ops & 2) && (ks * kSimtK) / kPad > (tj * kSimtTile) / kPad);
+  };
+  auto fetch = [&](const float* base, int tile, int ks, bool tr, int64_t ld_t) -> float4 {
+    return tr ? *reinterpret_cast<const float4*>(base + (int64_t)(ks * kSimtK + qk) * ld_t + tile * kSimtTile + qj)
+              : *reinterpret_cast<const float4*>(base + (int64_t)(tile * kSimtTile + lrow) * pb.Kp + ks * kSimtK + lk);
+  };
+  const int64_t ldt_p = pb.Kp, ldt_q = pb.q_mn ? pb.Np : pb.Kp;
   const int ksteps = (int)(pb.Kp / kSimtK);
-  float4 pa = *reinterpret_cast<const float4*>(P + (int64_t)lrow * pb.Kp + lk);
-  float4 qa = pb.q_mn ? *reinterpret_cast<const float4*>(Q + (int64_t)qk * pb.Np + qj)
-                      : *reinterpret_cast<const float4*>(Q + (int64_t)lrow * pb.Kp + lk);
+  float4 pa = fetch(P, ti, 0, p_transposed(0), ldt_p);
+  float4 qa = fetch(Q, tj, 0, q_transposed(0), ldt_q);
   for (int ks = 0; ks < ksteps; ++ks) {
-    As[lk + 0][lrow] = pa.x; As[lk + 1][lrow] = pa.y; As[lk + 2][lrow] = pa.z; As[lk + 3][lrow] = pa.w;
-    if (pb.q_mn) {
+    if (p_transposed(ks)) {
+      *reinterpret_cast<float4*>(&As[qk][qj]) = pa;
+    } else {
+      As[lk + 0][lrow] = pa.x; As[lk + 1][lrow] = pa.y; As[lk + 2][lrow] = pa.z; As[lk + 3][lrow] = pa.w;
+    }
+    if (q_transposed(ks)) {
       *reinterpret_cast<float4*>(&Bs[qk][qj]) = qa;
     } else {
       Bs[lk + 0][lrow] = qa.x; Bs[lk + 1][lrow] = qa.y; Bs[lk + 2][lrow] = qa.z; Bs[lk + 3][lrow] = qa.w;
     }
     __syncthreads();
     if (ks + 1 < ksteps) {
-      pa = *reinterpret_cast<const float4*>(P + (int64_t)lrow * pb.Kp + (ks + 1) * kSimtK + lk);
-      qa = pb.q_mn ? *reinterpret_cast<const float4*>(Q + (int64_t)((ks + 1) * kSimtK + qk) * pb.Np + qj)
-                   : *reinterpret_cast<const float4*>(Q + (int64_t)lrow * pb.Kp + (ks + 1) * kSimtK + lk);
+      pa = fetch(P, ti, ks + 1, p_transposed(ks + 1), ldt_p);
+      qa = fetch(Q, tj, ks + 1, q_transposed(ks + 1), ldt_q);
     }
 #pragma unroll
     for (int k = 0; k < kSimtK; ++k) {
@@ -93,7 +109,8 @@ gemm_simt_kernel(GemmProblem pb, Epilogue ep) {
 cudaError_t launch_gemm_simt(const GemmProblem& pb, const Epilogue& ep, cudaStream_t stream,
                              int64_t* launches) {
   const int64_t mt = pb.Mp / kSimtTile, nt = pb.Np / kSimtTile;
-  const int64_t tiles = pb.symmetric ? mt * (mt + 1) / 2 : mt * nt;
+  const int64_t nb = pb.Mp / kPad;
+  const int64_t tiles = pb.symmetric ? 4 * (nb * (nb + 1) / 2) : mt * nt;
   if (tiles > 0x7fffffffLL || pb.batch > 65535) return cudaErrorInvalidValue;
   *launches += 1;
   dim3 grid((unsigned)tiles, (unsigned)pb.batch, 1);

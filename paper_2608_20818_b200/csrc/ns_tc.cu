@@ -1,8 +1,11 @@
 // Tensor-core NS5 products for sm_100a: D[i,j] = sum_k P[i,k]*Q[j,k] with bf16
 // operands, fp32 accumulation in tensor memory, and the fused epilogues of
-// struct Epilogue (polynomial coefficients, Frobenius scale, mirror write of
-// the symmetric products, final parameter update).  Q may also be stored
-// [k][n] (N-major operand), which is how the update product reads X.
+// struct Epilogue (polynomial coefficients, Frobenius scale, final parameter
+// update).  Q may also be stored [k][n] (N-major operand), which is how the
+// update product reads X.  The symmetric matrices A and B exist only as their
+// 256x256 blocks on and below the diagonal: the products that consume them
+// read a missing block from its mirror image as an M/N-major operand, so no
+// product ever writes a transposed copy.
 //
 // Persistent CTA pairs (clusters of two CTAs on two SMs), 352 threads per CTA.
 // A pair computes a 256x256 tile with tcgen05.mma.cta_group::2: each CTA holds
@@ -16,10 +19,11 @@
 //   warps 2..9  epilogue arithmetic: two warps per TMEM lane quadrant; the
 //               tile is finished in four slabs of 64 columns.  Per slab:
 //               tcgen05.ld of the fp32 accumulator, auxiliary operand read
-//               from a shared-memory slab, result written back in place and,
-//               transposed, into a second slab
-//   warp 10     epilogue I/O: TMA load of the auxiliary slab, TMA stores of
-//               the result slab and of its transpose
+//               from a shared-memory slab, result written back in place (for
+//               the final update of a tall matrix: into the transposed
+//               parameter slab)
+//   warp 10     epilogue I/O: TMA loads of the auxiliary and parameter
+//               slabs, TMA stores of the result slab
 // All global traffic of the epilogues therefore moves as 128-byte swizzled
 // TMA boxes, the final parameter update included (the parameter tile is loaded
 // into the second slab, updated there and stored back; tall matrices use the
@@ -240,13 +244,23 @@ __device__ __forceinline__ TileCoord decode_tile(int t, int tiles_per_mat, int s
   return c;
 }
 
+// Q_MN and SYM_OPS are compile-time so that each product keeps a main loop
+// with constant descriptor strides (a run-time choice measurably slowed the
+// products that need none).
+template <int Q_MN, int SYM_OPS>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ,
                const __grid_constant__ CUtensorMap mapAux, const __grid_constant__ CUtensorMap mapDst,
-               const __grid_constant__ CUtensorMap mapDstT, int ktiles, int tiles_per_mat,
-               int total_tiles, int symmetric, int mt, int q_mn, Epilogue ep, int* status) {
+               const __grid_constant__ CUtensorMap mapDstT, const __grid_constant__ CUtensorMap mapSymT,
+               int ktiles, int tiles_per_mat, int total_tiles, int symmetric, int mt, Epilogue ep,
+               int* status) {
+  constexpr int q_mn = Q_MN, sym_ops = SYM_OPS;
   // q_mn: Q is stored [k][n] (n contiguous) instead of [n][k]; its tiles are
   // loaded as 64x64 boxes and consumed as an N-major MMA operand.
+  // sym_ops (bit 0: P, bit 1: Q): the operand is a symmetric matrix stored only
+  // in its 256x256 blocks on and below the diagonal.  A k-block right of the
+  // operand's diagonal block is read from the mirrored block, which holds it
+  // as [k][row]: 64x64 boxes through mapSymT, consumed as an M/N-major operand.
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* ebuf = smem + (size_t)kStages * kStageBytes;           // [kEpiBufs][kEpiBufBytes]
@@ -305,9 +319,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           // The leader's barrier counts the bytes of both CTAs' loads.
           if (rank == 0) mbar_expect_tx(&full[s], 2 * kStageBytes);
           const uint32_t lead_full = map_to_rank(&full[s], 0);
-          tma_load_3d_pair(sa, &mapP, lead_full, kt * kBK, c.ti * kBM, c.b);
+          const int kb = (kt * kBK) / kPad;                       // 256-block of this k-range
+          if ((sym_ops & 1) && kb > (c.ti >> 1)) {
+            tma_load_3d_pair(sa, &mapSymT, lead_full, c.ti * kBM, kt * kBK, c.b);
+            tma_load_3d_pair(sa + kBytesA / 2, &mapSymT, lead_full, c.ti * kBM + 64, kt * kBK, c.b);
+          } else {
+            tma_load_3d_pair(sa, &mapP, lead_full, kt * kBK, c.ti * kBM, c.b);
+          }
           const int n0 = c.tj * kBN + (int)rank * (kBN / 2);      // this CTA's 128 rows (columns) of Q
-          if (!q_mn) {
+          if ((sym_ops & 2) && kb > c.tj) {
+            tma_load_3d_pair(sa + kBytesA, &mapSymT, lead_full, n0, kt * kBK, c.b);
+            tma_load_3d_pair(sa + kBytesA + kBytesB / 2, &mapSymT, lead_full, n0 + 64, kt * kBK, c.b);
+          } else if (!q_mn) {
             tma_load_3d_pair(sa + kBytesA, &mapQ, lead_full, kt * kBK, n0, c.b);
           } else {
             tma_load_3d_pair(sa + kBytesA, &mapQ, lead_full, n0, kt * kBK, c.b);
@@ -334,6 +357,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
       uint32_t it = 0, acc_it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_it) {
+        const TileCoord c = decode_tile(t, tiles_per_mat, symmetric, mt);
         const int a = acc_it & 1;
         const uint32_t aph = (acc_it >> 1) & 1;
         if (!mbar_wait(&tempty[a], aph ^ 1, abort_flag, status)) break;
@@ -345,21 +369,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           if (!mbar_wait(&full[s], ph, abort_flag, status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
-          const uint64_t da = make_desc(sa);
-          if (!q_mn) {
-            const uint64_t db = make_desc(sa + kBytesA);
+          // K-major tile: 16 elements = 32 bytes further inside the swizzled row (+2 in 16-byte units);
+          // M/N-major tile: 16 k-rows = two 1024-byte atoms further (+128).
+          const int kb = (kt * kBK) / kPad;
+          const bool a_t = (sym_ops & 1) && kb > (c.ti >> 1);
+          const bool b_t = q_mn || ((sym_ops & 2) && kb > c.tj);
+          const uint64_t da = a_t ? make_desc_mn(sa) : make_desc(sa);
+          const uint64_t db = b_t ? make_desc_mn(sa + kBytesA) : make_desc(sa + kBytesA);
+          const uint32_t sa_k = a_t ? 128u : 2u, sb_k = b_t ? 128u : 2u;
+          const uint32_t idesc = kIdesc | (a_t ? (1u << 15) : 0u) | (b_t ? (1u << 16) : 0u);
 #pragma unroll
-            for (int k = 0; k < kBK / kUmmaK; ++k) {
-              // advance 16 elements = 32 bytes inside the swizzled row: +2 in 16-byte units
-              umma_bf16(tacc, da + 2 * k, db + 2 * k, kIdesc, (kt | k) != 0);
-            }
-          } else {
-            const uint64_t db = make_desc_mn(sa + kBytesA);
-#pragma unroll
-            for (int k = 0; k < kBK / kUmmaK; ++k) {
-              // Q: 16 k-rows = two 1024-byte atoms further: +128 in 16-byte units
-              umma_bf16(tacc, da + 2 * k, db + 128 * k, kIdesc | (1u << 16), (kt | k) != 0);
-            }
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            umma_bf16(tacc, da + sa_k * k, db + sb_k * k, idesc, (kt | k) != 0);
           }
           umma_commit_pair(&empty[s]);        // frees the stage in both CTAs when these MMAs have read it
         }
@@ -623,7 +644,13 @@ TcContext* tc_create(std::string* err) {
     return nullptr;
   }
   tc->sm_count = prop.multiProcessorCount;
-  ce = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (ce == cudaSuccess)
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (ce == cudaSuccess)
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (ce == cudaSuccess)
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce != cudaSuccess) {
     if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(ce);
     delete tc;
@@ -641,7 +668,7 @@ TcContext* tc_create(std::string* err) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n_clusters = 0;
-  ce = cudaOccupancyMaxActiveClusters(&n_clusters, gemm_tc_kernel, &cfg);
+  ce = cudaOccupancyMaxActiveClusters(&n_clusters, gemm_tc_kernel<0, 0>, &cfg);
   if (ce != cudaSuccess || n_clusters < 1) {
     if (err) *err = std::string("cudaOccupancyMaxActiveClusters: ") + cudaGetErrorString(ce);
     delete tc;
@@ -701,7 +728,7 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
                            cudaStream_t stream, int64_t* launches) {
   if (!tc) return cudaErrorInvalidValue;
   if (pb.Mp % kBN != 0 || pb.Np % kBN != 0 || pb.Kp % kBK != 0) return cudaErrorInvalidValue;
-  CUtensorMap mp, mq, maux, mdst, mdt;
+  CUtensorMap mp, mq, maux, mdst, mdt, msym;
   if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
   if (!pb.q_mn) {
     if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
@@ -711,7 +738,12 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   }
   // Epilogue maps (product epilogues only): auxiliary and result slabs of 128
   // rows x 64 columns, transposed result in boxes of 64 x 64.
-  maux = mp; mdst = mp; mdt = mp;
+  maux = mp; mdst = mp; mdt = mp; msym = mp;
+  if (pb.sym_ops) {
+    // 64x64 boxes over the symmetric operand (P; in the symmetric products Q is the same array)
+    if (pb.Mp != pb.Kp || ((pb.sym_ops & 2) && pb.Q != pb.P)) return cudaErrorInvalidValue;
+    if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, 64, &msym)) return cudaErrorInvalidValue;
+  }
   if (ep.aux && (ep.kind == 0 || ep.param_maps)) {
     if (ep.bs_aux != pb.Mp * ep.ld_aux) return cudaErrorInvalidValue;
     if (!get_map(tc, ep.aux, pb.Mp, ep.ld_aux, pb.batch, 128, &maux)) return cudaErrorInvalidValue;
@@ -749,8 +781,20 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel, mp, mq, maux, mdst, mdt, (int)(pb.Kp / kBK), (int)per_mat,
-                            (int)total, pb.symmetric, (int)mt, pb.q_mn, ep, status);
+  const int kt = (int)(pb.Kp / kBK);
+  if (pb.q_mn && pb.sym_ops == 1)
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<1, 1>, mp, mq, maux, mdst, mdt, msym, kt, (int)per_mat, (int)total,
+                              pb.symmetric, (int)mt, ep, status);
+  if (pb.q_mn && !pb.sym_ops)
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<1, 0>, mp, mq, maux, mdst, mdt, msym, kt, (int)per_mat, (int)total,
+                              pb.symmetric, (int)mt, ep, status);
+  if (!pb.q_mn && pb.sym_ops == 3)
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<0, 3>, mp, mq, maux, mdst, mdt, msym, kt, (int)per_mat, (int)total,
+                              pb.symmetric, (int)mt, ep, status);
+  if (!pb.q_mn && !pb.sym_ops)
+    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<0, 0>, mp, mq, maux, mdst, mdt, msym, kt, (int)per_mat, (int)total,
+                              pb.symmetric, (int)mt, ep, status);
+  return cudaErrorInvalidValue;   // no product of the recurrence needs another combination
 }
 
 }  // namespace prm

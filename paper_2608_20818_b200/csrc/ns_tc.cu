@@ -196,15 +196,11 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
       ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-// Arrives on the barrier at this offset in both CTAs of the pair once all MMAs
-// issued so far have completed.
-__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
-#pragma unroll
-  for (uint32_t r = 0; r < 2; ++r) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                 ::"r"(map_to_rank(bar, r))
-                 : "memory");
-  }
+// Arrives on the barrier at this shared::cluster address once all MMAs issued
+// so far have completed (issued once per CTA of the pair; no multicast form).
+__device__ __forceinline__ void umma_commit_to(uint32_t bar_cluster) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster)
+               : "memory");
 }
 // Issues the TMEM load; the registers are valid after tmem_ld_wait().
 __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
@@ -309,6 +305,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
+      const uint32_t lead_full0 = map_to_rank(&full[0], 0);
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         const TileCoord c = decode_tile(t, tiles_per_mat, symmetric, mt);
         for (int kt = 0; kt < ktiles; ++kt, ++it) {
@@ -318,7 +315,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           uint8_t* sa = smem + (size_t)s * kStageBytes;
           // The leader's barrier counts the bytes of both CTAs' loads.
           if (rank == 0) mbar_expect_tx(&full[s], 2 * kStageBytes);
-          const uint32_t lead_full = map_to_rank(&full[s], 0);
+          const uint32_t lead_full = lead_full0 + 8u * s;
           const int kb = (kt * kBK) / kPad;                       // 256-block of this k-range
           if ((sym_ops & 1) && kb > (c.ti >> 1)) {
             tma_load_3d_pair(sa, &mapSymT, lead_full, c.ti * kBM, kt * kBK, c.b);
@@ -354,8 +351,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0 && rank == 0) {
+      // This one thread feeds the tensor pipe of two SMs: everything that does
+      // not change per k-block is computed once (cluster addresses of the
+      // barriers, the constant halves of the descriptors).
       uint32_t it = 0, acc_it = 0;
       bool ok = true;
+      const uint32_t smem0 = smem_u32(smem);
+      const uint32_t empty_c0 = map_to_rank(&empty[0], 0), empty_c1 = map_to_rank(&empty[0], 1);
+      const uint32_t tfull_c0 = map_to_rank(&tfull[0], 0), tfull_c1 = map_to_rank(&tfull[0], 1);
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++acc_it) {
         const TileCoord c = decode_tile(t, tiles_per_mat, symmetric, mt);
         const int a = acc_it & 1;
@@ -368,7 +371,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           const uint32_t ph = (it / kStages) & 1;
           if (!mbar_wait(&full[s], ph, abort_flag, status)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t sa = smem_u32(smem + (size_t)s * kStageBytes);
+          const uint32_t sa = smem0 + (uint32_t)s * kStageBytes;
           // K-major tile: 16 elements = 32 bytes further inside the swizzled row (+2 in 16-byte units);
           // M/N-major tile: 16 k-rows = two 1024-byte atoms further (+128).
           const int kb = (kt * kBK) / kPad;
@@ -382,9 +385,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             umma_bf16(tacc, da + sa_k * k, db + sb_k * k, idesc, (kt | k) != 0);
           }
-          umma_commit_pair(&empty[s]);        // frees the stage in both CTAs when these MMAs have read it
+          umma_commit_to(empty_c0 + 8u * s);    // frees the stage in both CTAs when these MMAs have read it
+          umma_commit_to(empty_c1 + 8u * s);
         }
-        if (ok) umma_commit_pair(&tfull[a]);  // accumulator complete in both CTAs
+        if (ok) {                               // accumulator complete in both CTAs
+          umma_commit_to(tfull_c0 + 8u * a);
+          umma_commit_to(tfull_c1 + 8u * a);
+        }
       }
     }
   } else if (warp == kIoWarp) {

@@ -127,7 +127,7 @@ PRM_API int prm_step_h2d(prm_ctx* ctx, void* const* params, void* const* grads_d
 
 /*
  * The schedule and the shape grouping, without touching the device.
- *   is_refresh      1 iff step_idx mod K == 0
+ *   is_refresh      1 iff step_idx mod K == 0 (and PRM_OPT_NO_REFRESH is off)
  *   n_groups        number of distinct (rows, cols) pairs
  *   group_of_mat    [n_mats] group id, ids numbered by first appearance
  *   order_in_group  [n_mats] position inside the group, caller order kept

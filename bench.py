@@ -41,12 +41,18 @@ ROW_DRAM_BYTES_PER_ELEMENT = 14.0   # wide; the captures never exceed the algori
 
 
 # ----------------------------------------------------------------- accounting
-def ns5_flops(shapes):
-    """(executed with symmetry, paper model) flop of one refresh."""
+def ns5_flops(shapes, gram_iters=None):
+    """(executed, paper model) flop of one refresh.  Executed: the printed
+    recurrence with triangle-only symmetric products, 15r^2c+5r^3 per matrix, or
+    9r^2c+11r^3 where the library runs the first three iterations in Gram space
+    (gram_iters: {shape: 0 or 3}, as prm_group_info reports)."""
     ex = mo = 0
     for (m, n) in shapes:
         r, c = min(m, n), max(m, n)
-        ex += 15 * r * r * c + 5 * r ** 3
+        if gram_iters and gram_iters.get((m, n), 0):
+            ex += 9 * r * r * c + 11 * r ** 3
+        else:
+            ex += 15 * r * r * c + 5 * r ** 3
         mo += 20 * r * r * c + 10 * r ** 3
     return ex, mo
 
@@ -229,6 +235,8 @@ def main():
     ap.add_argument("--K", type=int, default=None)
     ap.add_argument("--check-mode", action="store_true", help="NS5 in fp32 on CUDA cores")
     ap.add_argument("--first-step", type=int, default=None, help="step index of the first warm-up step")
+    ap.add_argument("--printed-ns5", action="store_true",
+                    help="all five NS5 iterations as printed (no Gram-space iterations)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -258,7 +266,9 @@ def main():
     n = len(wl.shapes)
     io_bytes = 4 if wl.io_dtype == "fp32" else 2
     opt = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
-                                io_dtype=wl.io_dtype, check_mode=args.check_mode, device=dev)
+                                io_dtype=wl.io_dtype, check_mode=args.check_mode, gram_span=not args.printed_ns5,
+                                device=dev)
+    gram_iters = {(g["rows"], g["cols"]): g["gram_iters"] for g in opt.groups()}
     params = [make_param(wl, i, dev) for i in range(n)]
     moms = [make_momentum(wl, i, dev) for i in range(n)]
     # One gradient set per matrix kind and step parity keeps generation cheap;
@@ -347,11 +357,13 @@ def main():
     pk = peaks()
     amort = (mean_ref + (K - 1) * mean_row) / K if (ref_ms and (row_ms or K == 1)) else total_ms / args.steps
     n_ref, n_row = len(ref_ms), len(row_ms)
-    ex, mo = ns5_flops(wl.shapes)
+    ex, mo = ns5_flops(wl.shapes, gram_iters)
+    ex_printed, _ = ns5_flops(wl.shapes)
     el = elements(wl.shapes)
     row_bytes = el * (3 * io_bytes + 8)   # g and p read, p write (I/O dtype), m read and write (fp32)
-    gemm_ms = sum(prof[k][0] for k in ("gram", "poly", "update", "update_final"))
-    gemm_launches = sum(prof[k][1] for k in ("gram", "poly", "update", "update_final"))
+    gemm_classes = ("gram", "poly", "update", "update_final", "gramspace")
+    gemm_ms = sum(prof[k][0] for k in gemm_classes)
+    gemm_launches = sum(prof[k][1] for k in gemm_classes)
     row_kernel_ms = prof["row_wide"][0] + prof["row_tall"][0]
     out = {
         "metric": METRIC, "value": per_replica_ms(amort, world), "unit": "ms/step", "n_gpus": world, "steps": args.steps,
@@ -361,6 +373,9 @@ def main():
         "config": {"workload": wl.name, "K": K, "matrices": n, "blocks": wl.blocks, "d": wl.d,
                    "elements": el, "io_dtype": wl.io_dtype, "momentum_dtype": "fp32",
                    "ns5": "fp32 check mode" if args.check_mode else "bf16 tcgen05",
+                   "ns5_schedule": ("five iterations as printed" if not any(gram_iters.values()) else
+                                    "iterations 1-3 in Gram space for %d of %d matrices, 4-5 as printed" % (
+                                        sum(1 for sh in wl.shapes if gram_iters.get(tuple(sh), 0)), n)),
                    "replicas": world, "l2": "inputs larger than L2 (working set %.1f GB)" % (el * 8 / 1e9),
                    "first_timed_step_index": t_first + args.warmup},
         "refresh_ms": mean_ref if n_ref else None, "row_step_ms": mean_row if n_row else None,
@@ -378,6 +393,10 @@ def main():
     if n_ref and gemm_ms > 0:
         tf_exec = ex * n_ref / (gemm_ms * 1e-3) / 1e12
         out["ns5"] = {"TFLOP/s_exec": tf_exec, "TFLOP/s_model": mo * n_ref / (gemm_ms * 1e-3) / 1e12,
+                      # the printed recurrence's symmetric count over the same time: what a kernel that ran
+                      # all five iterations on X would have to sustain to be as fast
+                      "TFLOP/s_printed_equivalent": ex_printed * n_ref / (gemm_ms * 1e-3) / 1e12,
+                      "exec_flop_per_refresh": ex, "printed_flop_per_refresh": ex_printed,
                       "TFLOP/s_exec_whole_refresh": ex / (mean_ref * 1e-3) / 1e12,
                       "frac_of_measured_burst": tf_exec / pk["bf16_tflops"],
                       "frac_of_measured_sustained": tf_exec / pk["bf16_tflops_sustained"],

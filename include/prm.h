@@ -69,6 +69,18 @@ extern "C" {
 #define PRM_OPT_GAMMA_NS    10  /* multiplier on the NS5 branch, default 1 (the paper's method);
                                    "scalar-controlled" sets it to gamma */
 #define PRM_OPT_NO_REFRESH  11  /* 1: RowNorm at every step, no NS5 schedule; default 0 */
+/* How the tensor-core path evaluates the five NS5 iterations (Appendix "Cost of
+ * NS5").  The iteration X <- aX + BX with A = X X^T, B = bA + cA^2 keeps every A_k
+ * a polynomial in A_0, and A_{k+1} = (aI + B_k) A_k (aI + B_k).  1 (default): for
+ * matrices with at least 1024 oriented rows r and c >= 1.5 r columns the first
+ * three iterations work on r x r matrices only (A_1, A_2 and the product of the
+ * three factors aI + B_k from r x r products), then X_3 comes from one r x c
+ * product and the last two iterations run as printed: 9 r^2 c + 11 r^3 flop
+ * instead of 15 r^2 c + 5 r^3, the same result in exact arithmetic.  0: all five
+ * iterations as printed.  The check mode always runs them as printed.  Before
+ * set_workspace (the workspace holds two more r x r matrices per refreshed
+ * matrix when this is on). */
+#define PRM_OPT_NS_GRAM_SPAN 12
 
 
 
@@ -136,6 +148,16 @@ PRM_API int prm_step_h2d(prm_ctx* ctx, void* const* params, void* const* grads_d
 PRM_API int prm_plan(const prm_ctx* ctx, int64_t step_idx, int* is_refresh,
              int* n_groups, int* group_of_mat, int* order_in_group);
 
+/*
+ * One shape group of the plan (0 <= group < n_groups): its stored shape, the
+ * number of matrices, how many of them one refresh sub-batch holds with the
+ * current workspace cap, and how many leading NS5 iterations the refresh runs
+ * in Gram space (0 or 3, see PRM_OPT_NS_GRAM_SPAN).  Host only.  Any output
+ * pointer may be NULL.  PRM_ERR_ARG for a group out of range.
+ */
+PRM_API int prm_group_info(const prm_ctx* ctx, int group, int64_t* rows, int64_t* cols,
+                   int* count, int* ns_batch, int* gram_iters);
+
 /* Reads the device status word (synchronises the device first): PRM_OK, or
  * PRM_ERR_DEVICE_TIMEOUT if a kernel gave up on a bounded wait since the last
  * call; the word is cleared. */
@@ -174,7 +196,8 @@ PRM_API int64_t prm_launch_count(const prm_ctx* ctx);
 #define PRM_PROF_POLY          4  /* B = b A + c A^2 */
 #define PRM_PROF_UPDATE        5  /* X <- a X + B X */
 #define PRM_PROF_UPDATE_FINAL  6  /* last X update fused with the parameter update */
-#define PRM_PROF_COUNT         7
+#define PRM_PROF_GRAMSPACE     7  /* r x r products of the Gram-space iterations (PRM_OPT_NS_GRAM_SPAN) */
+#define PRM_PROF_COUNT         8
 PRM_API int prm_profile(prm_ctx* ctx, int enable);
 PRM_API int prm_profile_read(prm_ctx* ctx, double* ms, int64_t* launches, int n_classes);
 

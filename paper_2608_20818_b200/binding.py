@@ -37,16 +37,17 @@ PRM_OPT_WD = 8
 PRM_OPT_NS_WORKSPACE_BYTES = 9
 PRM_OPT_GAMMA_NS = 10
 PRM_OPT_NO_REFRESH = 11
+PRM_OPT_NS_GRAM_SPAN = 12
 
 EXPORTS = (
     "prm_create", "prm_set_option", "prm_workspace_bytes", "prm_set_workspace", "prm_step",
     "prm_step_h2d", "prm_plan", "prm_status", "prm_last_error", "prm_launch_count", "prm_destroy",
     "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc", "prm_selftest_timeout", "prm_adamw_step",
-    "prm_tall_shard_scratch_bytes", "prm_tall_shard_stats", "prm_tall_shard_apply",
+    "prm_tall_shard_scratch_bytes", "prm_tall_shard_stats", "prm_tall_shard_apply", "prm_group_info",
 )
 PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
-PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_COUNT = 4, 5, 6, 7
-PROF_NAMES = ("row_wide", "row_tall", "prepass", "gram", "poly", "update", "update_final")
+PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_GRAMSPACE, PRM_PROF_COUNT = 4, 5, 6, 7, 8
+PROF_NAMES = ("row_wide", "row_tall", "prepass", "gram", "poly", "update", "update_final", "gramspace")
 
 _lib_handle = None
 
@@ -82,6 +83,9 @@ def lib():
     L.prm_step_h2d.restype = c_int
     L.prm_plan.argtypes = [c_void_p, c_int64, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]
     L.prm_plan.restype = c_int
+    L.prm_group_info.argtypes = [c_void_p, c_int, POINTER(c_int64), POINTER(c_int64), POINTER(c_int), POINTER(c_int),
+                                 POINTER(c_int)]
+    L.prm_group_info.restype = c_int
     L.prm_status.argtypes = [c_void_p]
     L.prm_status.restype = c_int
     L.prm_last_error.argtypes = [c_void_p]
@@ -165,6 +169,16 @@ def prm_plan(h, step_idx, n_mats):
     return bool(is_refresh.value), n_groups.value, list(g), list(o)
 
 
+def prm_group_info(h, group):
+    """{rows, cols, count, ns_batch, gram_iters} of one shape group."""
+    rows, cols = c_int64(), c_int64()
+    count, ns_batch, gram_iters = c_int(), c_int(), c_int()
+    _check(lib().prm_group_info(h, int(group), byref(rows), byref(cols), byref(count), byref(ns_batch),
+                                byref(gram_iters)), h)
+    return {"rows": rows.value, "cols": cols.value, "count": count.value, "ns_batch": ns_batch.value,
+            "gram_iters": gram_iters.value}
+
+
 def prm_status(h):
     return int(lib().prm_status(h))
 
@@ -240,7 +254,7 @@ class PeriodicRowwiseMuon:
 
     def __init__(self, shapes, K, beta=0.95, nesterov=False, lr=5e-3, wd=0.01, *, gamma=0.15,
                  eps_row=1e-8, eps_ns=1e-7, scale_mode=1, io_dtype="bf16", check_mode=False,
-                 ns_workspace_bytes=None, gamma_ns=1.0, no_refresh=False, device="cuda"):
+                 ns_workspace_bytes=None, gamma_ns=1.0, no_refresh=False, gram_span=True, device="cuda"):
         self.shapes = [(int(m), int(n)) for (m, n) in shapes]
         self.device = torch.device(device)
         self.io_dtype = io_dtype
@@ -255,6 +269,7 @@ class PeriodicRowwiseMuon:
             prm_set_option(self.h, PRM_OPT_CHECK_MODE, 1 if check_mode else 0)
             prm_set_option(self.h, PRM_OPT_GAMMA_NS, gamma_ns)
             prm_set_option(self.h, PRM_OPT_NO_REFRESH, 1 if no_refresh else 0)
+            prm_set_option(self.h, PRM_OPT_NS_GRAM_SPAN, 1 if gram_span else 0)
             if ns_workspace_bytes is not None:
                 prm_set_option(self.h, PRM_OPT_NS_WORKSPACE_BYTES, ns_workspace_bytes)
             nbytes = prm_workspace_bytes(self.h)
@@ -302,6 +317,11 @@ class PeriodicRowwiseMuon:
 
     def plan(self, step_idx):
         return prm_plan(self.h, step_idx, len(self.shapes))
+
+    def groups(self):
+        """One dict per shape group (see prm_group_info)."""
+        n_groups = self.plan(0)[1]
+        return [prm_group_info(self.h, g) for g in range(n_groups)]
 
     def status(self):
         return prm_status(self.h)

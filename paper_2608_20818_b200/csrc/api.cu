@@ -25,6 +25,7 @@ struct prm_ctx {
   size_t ns_budget = (size_t)8 << 30;
   float gamma_ns = 1.f;   // multiplier on the NS5 branch (ablation: "scalar-controlled" uses gamma)
   int no_refresh = 0;     // ablation: RowNorm at every step
+  int gram_span = 1;      // first NS5 iterations in Gram space where it pays (tensor-core path)
 
   std::vector<Group> groups;
   std::vector<int> group_of_mat, order_in_group, slot_of_mat;   // slot = index in pointer tables
@@ -111,7 +112,12 @@ static void compute_layout(prm_ctx* c) {
       g.tall_scratch_off = off; off = align_up(off + (size_t)g.count * nblk * g.cols * 4, 256);
       g.tall_nu_off = off;      off = align_up(off + (size_t)g.count * g.cols * 4, 256);
     }
-    const size_t per_mat = e * (size_t)(2 * g.rp * g.cp + 2 * g.rp * g.rp);   // X ping-pong, A, B
+    // Gram-space iterations trade 6 r^2 (c - r) flop for six r^3 products: worth it
+    // from c = 1.5 r on; below 1024 rows the time is noise and the bf16 rounding of the
+    // small r x r matrices averages less well, so those stay on the printed recurrence.
+    g.gram_iters = (!c->check_mode && c->gram_span && g.rp >= 1024 && 2 * g.cp >= 3 * g.rp) ? kGramIters : 0;
+    // X ping-pong, A, B (+ two more r x r matrices for the Gram-space iterations)
+    const size_t per_mat = e * (size_t)(2 * g.rp * g.cp + (g.gram_iters ? 4 : 2) * g.rp * g.rp);
     int nb = (int)std::min<size_t>((size_t)g.count, std::max<size_t>(1, c->ns_budget / per_mat));
     // equal sub-batches: 42 matrices with room for 18 run as 14+14+14, not 18+18+6
     const int chunks = (g.count + nb - 1) / nb;
@@ -196,6 +202,7 @@ extern "C" int prm_set_option(prm_ctx* c, int key, double v) {
       c->no_refresh = (int)v; return PRM_OK;
     case PRM_OPT_IO_DTYPE:
     case PRM_OPT_CHECK_MODE:
+    case PRM_OPT_NS_GRAM_SPAN:
     case PRM_OPT_NS_WORKSPACE_BYTES:
       if (attached) return fail(c, PRM_ERR_STATE, "option must be set before prm_set_workspace");
       if (key == PRM_OPT_NS_WORKSPACE_BYTES) {
@@ -203,7 +210,7 @@ extern "C" int prm_set_option(prm_ctx* c, int key, double v) {
         c->ns_budget = (size_t)v;
       } else {
         if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
-        (key == PRM_OPT_IO_DTYPE ? c->io_fp32 : c->check_mode) = (int)v;
+        (key == PRM_OPT_IO_DTYPE ? c->io_fp32 : key == PRM_OPT_CHECK_MODE ? c->check_mode : c->gram_span) = (int)v;
       }
       compute_layout(c);
       return PRM_OK;
@@ -241,6 +248,18 @@ extern "C" int prm_plan(const prm_ctx* c, int64_t step_idx, int* is_refresh, int
   return PRM_OK;
 }
 
+extern "C" int prm_group_info(const prm_ctx* c, int group, int64_t* rows, int64_t* cols, int* count,
+                              int* ns_batch, int* gram_iters) {
+  if (!c || group < 0 || group >= (int)c->groups.size()) return PRM_ERR_ARG;
+  const Group& g = c->groups[group];
+  if (rows) *rows = g.rows;
+  if (cols) *cols = g.cols;
+  if (count) *count = g.count;
+  if (ns_batch) *ns_batch = g.ns_batch;
+  if (gram_iters) *gram_iters = g.gram_iters;
+  return PRM_OK;
+}
+
 static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepScalars s,
                          cudaStream_t stream) {
   const size_t e = c->check_mode ? 4 : 2;
@@ -252,8 +271,10 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
     const int nb = std::min(g.ns_batch, g.count - done);
     char* base = c->ws + c->off_ns;
     char* X[2] = {base, base + e * rc * nb};
-    char* A = base + 2 * e * rc * nb;
-    char* B = A + e * rr * nb;
+    char* R[4];                                      // r x r matrices (lower blocks)
+    for (int k = 0; k < 4; ++k) R[k] = base + 2 * e * rc * nb + (size_t)k * e * rr * nb;
+    char* A = R[0];
+    char* B = R[1];
     const int first = g.first + done;
     cudaError_t ce;
     {
@@ -267,8 +288,61 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
       return c->check_mode ? launch_gemm_simt(pb, ep, stream, &c->launches)
                            : launch_gemm_tc(c->tc, pb, ep, status, stream, &c->launches);
     };
-    int cur = 0;
-    for (int it = 0; it < kNsIters; ++it) {
+    int cur = 0, it0 = 0;
+    ce = cudaSuccess;
+    if (g.gram_iters) {
+      // The first three iterations without touching X (tensor-core path).  With
+      // P_k = aI + B_k, B_k = bA_k + cA_k^2, the recurrence reads X_{k+1} = P_k X_k
+      // and A_{k+1} = X_{k+1} X_{k+1}^T = P_k A_k P_k, all polynomials in A_0 and
+      // therefore symmetric and commuting.  So A_1, A_2 follow from r x r products,
+      // and X_3 = (P_2 P_1 P_0) X_0 = a^3 X_0 + Q X_0 needs one r x c product, where
+      // Q (the product without its a^3 I term, which stays an fp32 coefficient) is
+      // accumulated beside.  In exact arithmetic this is the printed recurrence;
+      // the last two iterations, whose rounding decides the error, run as printed.
+      auto sym = [&](const char* Pm, const char* Qm, float k_acc, const char* aux, float k_aux, const char* aux2,
+                     float k_aux2, char* dst, int cls) -> cudaError_t {
+        GemmProblem pb;
+        pb.P = Pm; pb.Q = Qm; pb.Mp = g.rp; pb.Np = g.rp; pb.Kp = g.rp;
+        pb.bs_P = rr; pb.bs_Q = rr; pb.batch = nb; pb.symmetric = 1; pb.sym_ops = 3;
+        Epilogue ep;
+        ep.k_acc = k_acc; ep.k_aux = k_aux; ep.aux = aux; ep.ld_aux = g.rp; ep.bs_aux = rr;
+        if (aux2) { ep.aux2 = aux2; ep.k_aux2 = k_aux2; ep.ld_aux2 = g.rp; ep.bs_aux2 = rr; }
+        ep.dst = dst; ep.ld_dst = g.rp; ep.bs_dst = rr;
+        return gemm(pb, ep, cls);
+      };
+      auto poly = [&](const char* Am, char* Bm) { return sym(Am, Am, kNsC, Am, kNsB, nullptr, 0.f, Bm, PRM_PROF_POLY); };
+      const float a = kNsA;
+      GemmProblem pa;
+      pa.P = X[0]; pa.Q = X[0]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
+      pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
+      Epilogue ea;
+      ea.dst = R[0]; ea.ld_dst = g.rp; ea.bs_dst = rr; ea.alpha = alpha; ea.alpha_pow = 2;
+      ce = gemm(pa, ea, PRM_PROF_GRAM);                                                          // A_0
+      if (ce == cudaSuccess) ce = poly(R[0], R[1]);                                              // B_0
+      if (ce == cudaSuccess) ce = sym(R[0], R[1], 1.f, R[0], a, nullptr, 0.f, R[2], PRM_PROF_GRAMSPACE);   // Z = A_0 P_0
+      if (ce == cudaSuccess) ce = sym(R[2], R[1], 1.f, R[2], a, nullptr, 0.f, R[0], PRM_PROF_GRAMSPACE);   // A_1 = Z P_0
+      if (ce == cudaSuccess) ce = poly(R[0], R[3]);                                              // B_1
+      if (ce == cudaSuccess)                                                                     // Q = P_1 P_0 - a^2 I
+        ce = sym(R[3], R[1], 1.f, R[1], a, R[3], a, R[2], PRM_PROF_GRAMSPACE);
+      if (ce == cudaSuccess) ce = sym(R[0], R[3], 1.f, R[0], a, nullptr, 0.f, R[1], PRM_PROF_GRAMSPACE);   // Z = A_1 P_1
+      if (ce == cudaSuccess) ce = sym(R[1], R[3], 1.f, R[1], a, nullptr, 0.f, R[0], PRM_PROF_GRAMSPACE);   // A_2 = Z P_1
+      if (ce == cudaSuccess) ce = poly(R[0], R[3]);                                              // B_2
+      if (ce == cudaSuccess)                                                                     // Q = P_2 P_1 P_0 - a^3 I
+        ce = sym(R[3], R[2], 1.f, R[2], a, R[3], a * a, R[1], PRM_PROF_GRAMSPACE);
+      if (ce == cudaSuccess) {                                                                   // X_3 = alpha (a^3 X_0 + Q X_0)
+        GemmProblem pu;
+        pu.P = R[1]; pu.Q = X[0]; pu.q_mn = 1; pu.sym_ops = 1; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
+        pu.bs_P = rr; pu.bs_Q = rc; pu.batch = nb; pu.symmetric = 0;
+        Epilogue eu;
+        eu.k_acc = 1.f; eu.k_aux = a * a * a; eu.aux = X[0]; eu.ld_aux = g.cp; eu.bs_aux = rc;
+        eu.alpha = alpha; eu.alpha_pow = 1;
+        eu.dst = X[1]; eu.ld_dst = g.cp; eu.bs_dst = rc;
+        ce = gemm(pu, eu, PRM_PROF_UPDATE);
+      }
+      cur = 1;
+      it0 = kGramIters;
+    }
+    for (int it = it0; it < kNsIters && ce == cudaSuccess; ++it) {
       // A = X X^T (times alpha^2 in the first iteration)
       GemmProblem pa;
       pa.P = X[cur]; pa.Q = X[cur]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;

@@ -19,6 +19,7 @@ constexpr float kNsA = 3.4445f;
 constexpr float kNsB = -4.7750f;
 constexpr float kNsC = 2.0315f;
 constexpr int kNsIters = 5;
+constexpr int kGramIters = 3;   // leading iterations that can run on the r x r Gram matrix alone
 
 // NS5 operands live in the workspace padded to multiples of kPad in both
 // dimensions; the padding is zero and stays zero through the recurrence.
@@ -147,6 +148,7 @@ struct Group {
   int64_t r = 0, c = 0;         // oriented shape, r <= c
   int64_t rp = 0, cp = 0;       // padded oriented shape (NS5 workspace)
   int ns_batch = 1;             // matrices refreshed per sub-batch
+  int gram_iters = 0;           // leading NS5 iterations run in Gram space (0 or kGramIters)
   size_t tall_scratch_off = 0;  // byte offset of column partials (tall groups)
   size_t tall_nu_off = 0;       // byte offset of column norms (tall groups)
 };

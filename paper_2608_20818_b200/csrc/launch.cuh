@@ -8,6 +8,8 @@ namespace prm {
 // Epilogue of every NS5 product D[i,j] = sum_k P[i,k]*Q[j,k].  With
 // f = alpha[b]^alpha_pow (1 if alpha is null) and
 // v = f*(k_acc*D[i,j] + k_aux*aux[i,j]):
+// (plus f*k_aux2*aux2[i,j] where a second auxiliary operand is given: the
+// Gram-space products of the tensor-core path)
 //   kind 0: dst[i,j] = v; if dst_t is set, dst_t[j,i] = v as well.  The
 //           symmetric products store only the blocks they compute (on and
 //           below the diagonal); their consumers read the mirrored block
@@ -21,6 +23,9 @@ struct Epilogue {
   int alpha_pow = 0;
   const void* aux = nullptr;      // [batch][Mp][ld_aux]
   int64_t ld_aux = 0, bs_aux = 0;
+  const void* aux2 = nullptr;     // [batch][Mp][ld_aux2], tensor-core path, kind 0 only
+  float k_aux2 = 0.f;
+  int64_t ld_aux2 = 0, bs_aux2 = 0;
   void* dst = nullptr;            // [batch][Mp][ld_dst]
   int64_t ld_dst = 0, bs_dst = 0;
   void* dst_t = nullptr;          // [batch][Np][ld_dst_t]
@@ -38,8 +43,8 @@ struct Epilogue {
 };
 
 // One batched product.  P: [batch][Mp][Kp], Q: [batch][Np][Kp]; Mp, Np, Kp
-// are multiples of kPad.  symmetric != 0: P == Q and only tiles of the lower
-// triangle are computed, the rest is filled by the mirror write.
+// are multiples of kPad.  symmetric != 0: the result is symmetric and only its
+// 256x256 blocks on and below the diagonal are computed and stored.
 struct GemmProblem {
   const void* P = nullptr;
   const void* Q = nullptr;
@@ -50,6 +55,8 @@ struct GemmProblem {
   int q_mn = 0;                   // Q is stored [batch][Kp][Np] (n contiguous) instead of [batch][Np][Kp]
   // Bit 0: P, bit 1: Q is a symmetric matrix of which only the 256x256 blocks on
   // and below the diagonal are stored; the rest is read from the mirrored block.
+  // P and Q may be two different symmetric matrices (symmetric != 0 then
+  // computes the lower blocks of P*Q, which is symmetric when they commute).
   int sym_ops = 0;
 };
 

@@ -243,20 +243,24 @@ __device__ __forceinline__ TileCoord decode_tile(int t, int tiles_per_mat, int s
 // Q_MN and SYM_OPS are compile-time so that each product keeps a main loop
 // with constant descriptor strides (a run-time choice measurably slowed the
 // products that need none).
-template <int Q_MN, int SYM_OPS>
+template <int Q_MN, int SYM_OPS, int AUX2>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ,
-               const __grid_constant__ CUtensorMap mapAux, const __grid_constant__ CUtensorMap mapDst,
-               const __grid_constant__ CUtensorMap mapDstT, const __grid_constant__ CUtensorMap mapSymT,
+               const __grid_constant__ CUtensorMap mapAux, const __grid_constant__ CUtensorMap mapAux2,
+               const __grid_constant__ CUtensorMap mapDst, const __grid_constant__ CUtensorMap mapDstT,
+               const __grid_constant__ CUtensorMap mapSymP, const __grid_constant__ CUtensorMap mapSymQ,
                int ktiles, int tiles_per_mat, int total_tiles, int symmetric, int mt, Epilogue ep,
                int* status) {
   constexpr int q_mn = Q_MN, sym_ops = SYM_OPS;
+  // AUX2: a second auxiliary operand (Epilogue::aux2) travels in the half of
+  // the slab buffer that the transposed result or the parameter tile would
+  // use; only the Gram-space products of two symmetric matrices need it.
   // q_mn: Q is stored [k][n] (n contiguous) instead of [n][k]; its tiles are
   // loaded as 64x64 boxes and consumed as an N-major MMA operand.
   // sym_ops (bit 0: P, bit 1: Q): the operand is a symmetric matrix stored only
   // in its 256x256 blocks on and below the diagonal.  A k-block right of the
   // operand's diagonal block is read from the mirrored block, which holds it
-  // as [k][row]: 64x64 boxes through mapSymT, consumed as an M/N-major operand.
+  // as [k][row]: 64x64 boxes through mapSymP / mapSymQ, consumed as an M/N-major operand.
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   uint8_t* ebuf = smem + (size_t)kStages * kStageBytes;           // [kEpiBufs][kEpiBufBytes]
@@ -318,15 +322,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           const uint32_t lead_full = lead_full0 + 8u * s;
           const int kb = (kt * kBK) / kPad;                       // 256-block of this k-range
           if ((sym_ops & 1) && kb > (c.ti >> 1)) {
-            tma_load_3d_pair(sa, &mapSymT, lead_full, c.ti * kBM, kt * kBK, c.b);
-            tma_load_3d_pair(sa + kBytesA / 2, &mapSymT, lead_full, c.ti * kBM + 64, kt * kBK, c.b);
+            tma_load_3d_pair(sa, &mapSymP, lead_full, c.ti * kBM, kt * kBK, c.b);
+            tma_load_3d_pair(sa + kBytesA / 2, &mapSymP, lead_full, c.ti * kBM + 64, kt * kBK, c.b);
           } else {
             tma_load_3d_pair(sa, &mapP, lead_full, kt * kBK, c.ti * kBM, c.b);
           }
           const int n0 = c.tj * kBN + (int)rank * (kBN / 2);      // this CTA's 128 rows (columns) of Q
           if ((sym_ops & 2) && kb > c.tj) {
-            tma_load_3d_pair(sa + kBytesA, &mapSymT, lead_full, n0, kt * kBK, c.b);
-            tma_load_3d_pair(sa + kBytesA + kBytesB / 2, &mapSymT, lead_full, n0 + 64, kt * kBK, c.b);
+            tma_load_3d_pair(sa + kBytesA, &mapSymQ, lead_full, n0, kt * kBK, c.b);
+            tma_load_3d_pair(sa + kBytesA + kBytesB / 2, &mapSymQ, lead_full, n0 + 64, kt * kBK, c.b);
           } else if (!q_mn) {
             tma_load_3d_pair(sa + kBytesA, &mapQ, lead_full, kt * kBK, n0, c.b);
           } else {
@@ -409,8 +413,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           const TileCoord c = decode_tile(blockIdx.x + (int)(g / kSlabs) * gridDim.x, tiles_per_mat, symmetric, mt);
           const int j0 = c.tj * kBN + (int)(g % kSlabs) * kSlabCols;
           uint8_t* buf = ebuf + (size_t)bsel * kEpiBufBytes;
-          mbar_expect_tx(&eready[bsel], (has_aux ? kSlabBytes : 0u) + (fin ? kSlabBytes : 0u));
+          mbar_expect_tx(&eready[bsel], (has_aux ? kSlabBytes : 0u) + ((fin || AUX2) ? kSlabBytes : 0u));
           if (has_aux) tma_load_3d(buf, &mapAux, &eready[bsel], j0, c.ti * kBM, c.b);
+          if (AUX2) tma_load_3d(buf + kSlabBytes, &mapAux2, &eready[bsel], j0, c.ti * kBM, c.b);
           if (fin) {
             // Parameter tile into the second slab: as stored (wide), or the
             // transposed region in two 64x64 boxes (tall).  Out-of-range parts read as zero.
@@ -486,6 +491,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
         const float al = ep.alpha ? ep.alpha[c.b] : 1.f;
         const float f = ep.alpha_pow == 2 ? al * al : (ep.alpha_pow == 1 ? al : 1.f);
         const float ka = f * ep.k_acc, kx = f * ep.k_aux;
+        const float kx2 = AUX2 ? f * ep.k_aux2 : 0.f;
         const bool write_t = c.mirror && ep.dst_t != nullptr;
 #pragma unroll 1
         for (int sl = 0; sl < kSlabs; ++sl, ++g) {
@@ -542,11 +548,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
             }
             int4 outv;
             __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(&outv);
+            if (AUX2) {
+              const int4 raw2 = *reinterpret_cast<const int4*>(buf + kSlabBytes + sw128(row, half * 4 + v));
+              const __nv_bfloat162* g2 = reinterpret_cast<const __nv_bfloat162*>(&raw2);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const float v0 = ka * __uint_as_float(r[8 * v + 2 * k]) + kx * x[2 * k];
-              const float v1 = ka * __uint_as_float(r[8 * v + 2 * k + 1]) + kx * x[2 * k + 1];
-              o2[k] = __floats2bfloat162_rn(v0, v1);
+              for (int k = 0; k < 4; ++k) {
+                const float2 yy = __bfloat1622float2(g2[k]);
+                const float v0 = ka * __uint_as_float(r[8 * v + 2 * k]) + (kx * x[2 * k] + kx2 * yy.x);
+                const float v1 = ka * __uint_as_float(r[8 * v + 2 * k + 1]) + (kx * x[2 * k + 1] + kx2 * yy.y);
+                o2[k] = __floats2bfloat162_rn(v0, v1);
+              }
+            } else {
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float v0 = ka * __uint_as_float(r[8 * v + 2 * k]) + kx * x[2 * k];
+                const float v1 = ka * __uint_as_float(r[8 * v + 2 * k + 1]) + kx * x[2 * k + 1];
+                o2[k] = __floats2bfloat162_rn(v0, v1);
+              }
             }
             *p = outv;
             if (write_t) {
@@ -651,13 +669,15 @@ TcContext* tc_create(std::string* err) {
     return nullptr;
   }
   tc->sm_count = prop.multiProcessorCount;
-  ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce == cudaSuccess)
-    ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 3, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce == cudaSuccess)
-    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 3, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce == cudaSuccess)
-    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (ce == cudaSuccess)
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce != cudaSuccess) {
     if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(ce);
     delete tc;
@@ -675,7 +695,7 @@ TcContext* tc_create(std::string* err) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n_clusters = 0;
-  ce = cudaOccupancyMaxActiveClusters(&n_clusters, gemm_tc_kernel<0, 0>, &cfg);
+  ce = cudaOccupancyMaxActiveClusters(&n_clusters, gemm_tc_kernel<0, 0, 0>, &cfg);
   if (ce != cudaSuccess || n_clusters < 1) {
     if (err) *err = std::string("cudaOccupancyMaxActiveClusters: ") + cudaGetErrorString(ce);
     delete tc;
@@ -735,7 +755,7 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
                            cudaStream_t stream, int64_t* launches) {
   if (!tc) return cudaErrorInvalidValue;
   if (pb.Mp % kBN != 0 || pb.Np % kBN != 0 || pb.Kp % kBK != 0) return cudaErrorInvalidValue;
-  CUtensorMap mp, mq, maux, mdst, mdt, msym;
+  CUtensorMap mp, mq, maux, maux2, mdst, mdt, msp, msq;
   if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
   if (!pb.q_mn) {
     if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
@@ -745,15 +765,23 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   }
   // Epilogue maps (product epilogues only): auxiliary and result slabs of 128
   // rows x 64 columns, transposed result in boxes of 64 x 64.
-  maux = mp; mdst = mp; mdt = mp; msym = mp;
-  if (pb.sym_ops) {
-    // 64x64 boxes over the symmetric operand (P; in the symmetric products Q is the same array)
-    if (pb.Mp != pb.Kp || ((pb.sym_ops & 2) && pb.Q != pb.P)) return cudaErrorInvalidValue;
-    if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, 64, &msym)) return cudaErrorInvalidValue;
+  maux = mp; maux2 = mp; mdst = mp; mdt = mp; msp = mp; msq = mp;
+  // 64x64 boxes over a symmetric operand, through which its mirrored blocks are read
+  if (pb.sym_ops & 1) {
+    if (pb.Mp != pb.Kp || !get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, 64, &msp)) return cudaErrorInvalidValue;
+  }
+  if (pb.sym_ops & 2) {
+    if (pb.Np != pb.Kp || pb.q_mn || !get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, 64, &msq)) return cudaErrorInvalidValue;
   }
   if (ep.aux && (ep.kind == 0 || ep.param_maps)) {
     if (ep.bs_aux != pb.Mp * ep.ld_aux) return cudaErrorInvalidValue;
     if (!get_map(tc, ep.aux, pb.Mp, ep.ld_aux, pb.batch, 128, &maux)) return cudaErrorInvalidValue;
+  }
+  if (ep.aux2) {
+    // second auxiliary operand: product epilogues of two symmetric operands only
+    if (ep.kind != 0 || !ep.aux || ep.dst_t || pb.q_mn || pb.sym_ops != 3) return cudaErrorInvalidValue;
+    if (ep.bs_aux2 != pb.Mp * ep.ld_aux2) return cudaErrorInvalidValue;
+    if (!get_map(tc, ep.aux2, pb.Mp, ep.ld_aux2, pb.batch, 128, &maux2)) return cudaErrorInvalidValue;
   }
   if (ep.kind == 0) {
     if (ep.bs_dst != pb.Mp * ep.ld_dst) return cudaErrorInvalidValue;
@@ -789,18 +817,15 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   const int kt = (int)(pb.Kp / kBK);
-  if (pb.q_mn && pb.sym_ops == 1)
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<1, 1>, mp, mq, maux, mdst, mdt, msym, kt, (int)per_mat, (int)total,
-                              pb.symmetric, (int)mt, ep, status);
-  if (pb.q_mn && !pb.sym_ops)
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<1, 0>, mp, mq, maux, mdst, mdt, msym, kt, (int)per_mat, (int)total,
-                              pb.symmetric, (int)mt, ep, status);
-  if (!pb.q_mn && pb.sym_ops == 3)
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<0, 3>, mp, mq, maux, mdst, mdt, msym, kt, (int)per_mat, (int)total,
-                              pb.symmetric, (int)mt, ep, status);
-  if (!pb.q_mn && !pb.sym_ops)
-    return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<0, 0>, mp, mq, maux, mdst, mdt, msym, kt, (int)per_mat, (int)total,
-                              pb.symmetric, (int)mt, ep, status);
+#define PRM_TC_LAUNCH(QMN, SYM, AX2)                                                                              \
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<QMN, SYM, AX2>, mp, mq, maux, maux2, mdst, mdt, msp, msq, kt,     \
+                            (int)per_mat, (int)total, pb.symmetric, (int)mt, ep, status)
+  if (pb.q_mn && pb.sym_ops == 1) PRM_TC_LAUNCH(1, 1, 0);
+  if (pb.q_mn && !pb.sym_ops) PRM_TC_LAUNCH(1, 0, 0);
+  if (!pb.q_mn && pb.sym_ops == 3 && ep.aux2) PRM_TC_LAUNCH(0, 3, 1);
+  if (!pb.q_mn && pb.sym_ops == 3) PRM_TC_LAUNCH(0, 3, 0);
+  if (!pb.q_mn && !pb.sym_ops) PRM_TC_LAUNCH(0, 0, 0);
+#undef PRM_TC_LAUNCH
   return cudaErrorInvalidValue;   // no product of the recurrence needs another combination
 }
 

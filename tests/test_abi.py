@@ -95,3 +95,30 @@ def test_workspace_scales_with_options():
     B.prm_set_option(h, B.PRM_OPT_NS_WORKSPACE_BYTES, 1)
     assert B.prm_workspace_bytes(h) < check
     B.prm_destroy(h)
+
+
+def test_group_info_and_gram_span_option():
+    shapes = [(2048, 6144), (2048, 2048), (8192, 2048), (2048, 6144), (256, 1024), (1024, 1280)]
+    h = B.prm_create(shapes, 5, 0.95, True, 1e-3, 0.0)
+    _, n_groups, group_of_mat, _ = B.prm_plan(h, 0, len(shapes))
+    assert n_groups == 5 and group_of_mat == [0, 1, 2, 0, 3, 4]
+    info = [B.prm_group_info(h, g) for g in range(n_groups)]
+    assert [(g["rows"], g["cols"], g["count"]) for g in info] == [
+        (2048, 6144, 2), (2048, 2048, 1), (8192, 2048, 1), (256, 1024, 1), (1024, 1280, 1)]
+    # Gram-space iterations: >= 1024 oriented rows and c >= 1.5 r (padded to 256)
+    assert [g["gram_iters"] for g in info] == [3, 0, 3, 0, 0]
+    assert all(g["ns_batch"] == g["count"] for g in info)
+    with_span = B.prm_workspace_bytes(h)
+    B.prm_set_option(h, B.PRM_OPT_NS_GRAM_SPAN, 0)
+    assert [B.prm_group_info(h, g)["gram_iters"] for g in range(n_groups)] == [0] * 5
+    assert B.prm_workspace_bytes(h) < with_span
+    B.prm_set_option(h, B.PRM_OPT_NS_GRAM_SPAN, 1)
+    B.prm_set_option(h, B.PRM_OPT_CHECK_MODE, 1)          # the check mode runs the printed recurrence
+    assert [B.prm_group_info(h, g)["gram_iters"] for g in range(n_groups)] == [0] * 5
+    with pytest.raises(B.PrmError) as e:
+        B.prm_set_option(h, B.PRM_OPT_NS_GRAM_SPAN, 2)
+    assert e.value.code == B.PRM_ERR_ARG
+    with pytest.raises(B.PrmError) as e:
+        B.prm_group_info(h, n_groups)
+    assert e.value.code == B.PRM_ERR_ARG
+    B.prm_destroy(h)

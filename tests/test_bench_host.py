@@ -28,6 +28,10 @@ def test_accounting_matches_the_shape_sets():
         ex, mo = bench.ns5_flops(wl.shapes)
         assert mo == 410 * d ** 3 * blocks          # 70 + 30 + 90 + 90 + 130 per block
         assert ex == 295 * d ** 3 * blocks          # 50 + 20 + 65 + 65 + 95 per block
+        # first three iterations in Gram space wherever c >= 1.5 r: 9 r^2 c + 11 r^3
+        span = {sh: (3 if max(sh) >= 1.5 * min(sh) else 0) for sh in set(map(tuple, wl.shapes))}
+        ex_span, mo_span = bench.ns5_flops(wl.shapes, span)
+        assert mo_span == mo and ex_span == 217 * d ** 3 * blocks   # 38 + 20 + 47 + 47 + 65 per block
     ex, mo = bench.ns5_flops(workload(4).shapes)
     assert abs(ex / 1e12 - 851.4) < 0.1 and abs(mo / 1e12 - 1183.3) < 0.1
     assert abs(14 * bench.elements(workload(4).shapes) / 1e9 - 177.6) < 0.1

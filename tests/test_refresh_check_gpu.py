@@ -15,13 +15,13 @@ pytestmark = pytest.mark.gpu
 SHAPES = [(256, 1024), (24, 40), (40, 24), (300, 520), (512, 256), (5, 5), (1, 9), (130, 1000), (768, 768)]
 
 
-def _direction_case(shapes, io, check_mode, seed, nesterov=True, ns_ws=None):
+def _direction_case(shapes, io, check_mode, seed, nesterov=True, ns_ws=None, gram_span=True):
     """W = 0, lr = 1, wd = 0: the step writes -s * NS5 direction."""
     cfg = U.oracle_cfg(K=3, beta=0.95, nesterov=nesterov, lr=1.0, wd=0.0, scale_mode=0)
     W, G, M = U.make_inputs(shapes, seed, io, grad_std=1e-3, mom_std=1e-3)
     for w in W:
         w.zero_()
-    Wg, Mg = U.gpu_step(shapes, W, G, M, 3, cfg, io, check_mode, ns_workspace_bytes=ns_ws)
+    Wg, Mg = U.gpu_step(shapes, W, G, M, 3, cfg, io, check_mode, ns_workspace_bytes=ns_ws, gram_span=gram_span)
     errs = []
     for i in range(len(shapes)):
         Wr, Mr = O.step_matrix(U.to_np64(W[i]), U.to_np64(G[i]), U.to_np64(M[i]), 3, cfg)

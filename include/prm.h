@@ -287,6 +287,70 @@ PRM_API int prm_tall_shard_apply(void* param_shard, const void* grad_shard, cons
                                  float lr, float wd, float gamma, float eps_row, float scale,
                                  const float* colsumsq, void* cuda_stream);
 
+/*
+ * Refresh over row shards: the bucketed all-gather pipeline (Section 3.3,
+ * "Distributed Execution"; Algorithm 2 lines 1-7; appendix "Idealized overlap
+ * model").  Every stored matrix is split over `world` ranks by rows as
+ * torch.chunk splits dim 0: chunk = ceil(rows / world), rank q owns rows
+ * [q*chunk, min(rows, (q+1)*chunk)) (possibly none).  The Muon matrices are
+ * partitioned into communication buckets; per bucket every rank fills one
+ * SEGMENT of bf16 elements, the segments are all-gathered (by the caller:
+ * NCCL or any other transport), and every rank then refreshes the bucket's
+ * full matrices and updates its own rows.  While one bucket is refreshed the
+ * next one is gathered.  The library does the device work on both sides of
+ * the exchange and the planning; it contains no communication.
+ *
+ * prm_shard_rows     the row range of one rank (host).
+ * prm_bucket_plan    host.  Walks the matrices in caller order; matrix i
+ *   reserves ceil8(chunk_i * cols_i) elements in every rank's segment
+ *   (offset_in_segment[i], a multiple of 8); a new bucket starts when the
+ *   gathered payload world * 2 bytes * segment would exceed bucket_bytes (a
+ *   bucket always holds at least one matrix).  Outputs: bucket_of_mat[n_mats],
+ *   offset_in_segment[n_mats], *n_buckets, segment_elems[b] for b < *n_buckets
+ *   (array of n_mats entries).
+ * prm_shard_momentum_pack   device.  Algorithm 1 line 2 on this rank's rows of
+ *   one matrix (momentum_shard updated in place) and the direction input U
+ *   (M_t, or beta*M_t + (1-beta)*G_t with nesterov) rounded to bf16 into
+ *   u_out, which points at the matrix's place in this rank's segment;
+ *   reserved_elems >= rows_local*cols elements are written, the tail as
+ *   zeros.  grad bf16 (io_fp32 = 0) or fp32; pointers 16-byte aligned.
+ *   bf16 is what the single-GPU refresh feeds NS5 as well, so sharding does
+ *   not change the NS5 input.
+ * prm_refresh_gathered      device, on a handle created over the GLOBAL
+ *   shapes with a workspace attached.  mats[k] (k < n): indices, in the
+ *   handle's matrix order, of the bucket's matrices; gathered: the all-gather
+ *   result, world segments of segment_elems bf16 elements, rank q's at
+ *   q*segment_elems; offsets[k]: offset_in_segment of mats[k];
+ *   param_shards[k]: this rank's rows of parameter mats[k] (bf16 or fp32 per
+ *   PRM_OPT_IO_DTYPE; may be NULL when the rank owns no row).  Per shape
+ *   group and sub-batch: the full oriented matrices are rebuilt from the
+ *   segments straight into the NS5 workspace (with the Frobenius norm), NS5
+ *   runs as in prm_step, and W_shard <- (1 - lr*wd) W_shard - lr*s(W)*X_5 is
+ *   applied to rows [row_start, row_start + row_count) only; s(W) uses the
+ *   global shape.  The gathered buffer may be reused as soon as the call's
+ *   work on cuda_stream has passed the rebuild of its last sub-batch, i.e.
+ *   after the call's work completes.  mats, offsets and param_shards are HOST
+ *   arrays.  Errors as for prm_step; PRM_ERR_SHAPE if a matrix does not fit
+ *   its segment.
+ * prm_pipeline_model  host.  Ideal two-stage pipeline over n_buckets buckets
+ *   with all-gather times a[l] and compute times c[l] (Eq. app-pipeline-time,
+ *   Eq. app-exposed-communication):
+ *     t_pipe = a[0] + sum_{l < n-1} max(c[l], a[l+1]) + c[n-1]
+ *     t_comm_exposed = a[0] + sum_{l < n-1} max(0, a[l+1] - c[l])
+ */
+PRM_API int prm_shard_rows(int64_t rows, int world, int rank, int64_t* row_start, int64_t* row_count);
+PRM_API int prm_bucket_plan(const int64_t* shapes, int n_mats, int world, int64_t bucket_bytes,
+                            int* bucket_of_mat, int64_t* offset_in_segment, int* n_buckets,
+                            int64_t* segment_elems);
+PRM_API int prm_shard_momentum_pack(const void* grad_shard, float* momentum_shard, int64_t rows_local,
+                                    int64_t cols, int64_t reserved_elems, int io_fp32, float beta,
+                                    int nesterov, void* u_out, void* cuda_stream);
+PRM_API int prm_refresh_gathered(prm_ctx* ctx, const int* mats, int n, const void* gathered,
+                                 int64_t segment_elems, const int64_t* offsets, int world, int rank,
+                                 void* const* param_shards, void* cuda_stream);
+PRM_API int prm_pipeline_model(const double* a, const double* c, int n_buckets, double* t_pipe,
+                               double* t_comm_exposed);
+
 /* Frees host resources.  Device memory belongs to the caller. */
 PRM_API int prm_destroy(prm_ctx* ctx);
 

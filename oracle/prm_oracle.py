@@ -31,7 +31,9 @@ Readings of the paper taken here (the paper is silent or ambiguous on them):
 Functions with a pin (tests/test_oracle_pins.py): momentum_update,
 direction_input, orient, orient_inv, rownorm, ns5, is_refresh,
 group_by_shape, step_matrix (decay term, learning-rate scaling, branch
-selection, gamma placement).
+selection, gamma placement), shard_rows (torch.chunk), pipeline_time (event
+simulation), refresh_from_shards (equals the dense step), bucket_plan (plan
+invariants only: the paper gives no bucketing rule, parity unpinned).
 """
 
 from __future__ import annotations
@@ -231,3 +233,70 @@ def adamw_step(p, g, m, v, t, lr=1e-4, beta1=0.9, beta2=0.95, eps=1e-8, wd=0.01)
     v_hat = v / (1.0 - beta2 ** t)
     p = p - lr * m_hat / (np.sqrt(v_hat) + eps)
     return p, m, v
+
+
+# --------------------------------------------------------------------------
+# Distributed execution of the refresh branch (Section 3.3; Algorithm 2 lines
+# 1-7; appendix "Idealized overlap model").  Host-side planning and the
+# reference result of a refresh computed from row shards.
+#
+# Readings taken here (the paper only says that the Muon matrices are
+# partitioned into communication buckets and that FSDP2 shards dim 0):
+# * rows are split as torch.chunk splits them, chunk = ceil(rows / world);
+# * buckets are filled greedily in the given matrix order, a matrix is never
+#   split, and a bucket is closed when the gathered payload (world segments of
+#   2-byte elements) would exceed the byte cap; every matrix's slot in a
+#   segment is rounded up to 8 elements.  Parity unpinned against the paper
+#   (it gives no rule); pinned by the invariants every valid plan must have.
+
+
+def shard_rows(rows, world, rank):
+    """(start, count) of rank's rows under dim-0 sharding (Section 3.3)."""
+    chunk = -(-rows // world)
+    lo = min(rows, rank * chunk)
+    hi = min(rows, lo + chunk)
+    return lo, hi - lo
+
+
+def bucket_plan(shapes, world, bucket_bytes):
+    """Communication buckets B_l of Algorithm 2: (bucket_of_mat, offset_in_segment, segment_elems)."""
+    bucket_of_mat, offsets, segments = [], [], []
+    seg = 0
+    for (m, n) in shapes:
+        chunk = -(-m // world)
+        need = -(-(chunk * n) // 8) * 8
+        if seg > 0 and (seg + need) * 2 * world > bucket_bytes:
+            segments.append(seg)
+            seg = 0
+        bucket_of_mat.append(len(segments))
+        offsets.append(seg)
+        seg += need
+    segments.append(seg)
+    return bucket_of_mat, offsets, segments
+
+
+def pipeline_time(a, c):
+    """(T_pipe, T_comm_exposed) of the ideal two-stage pipeline over buckets with
+    all-gather times a_l and compute times c_l (Eq. app-pipeline-time and
+    Eq. app-exposed-communication)."""
+    B = len(a)
+    t_pipe = a[0] + sum(max(c[l], a[l + 1]) for l in range(B - 1)) + c[B - 1]
+    t_exposed = a[0] + sum(max(0.0, a[l + 1] - c[l]) for l in range(B - 1))
+    return t_pipe, t_exposed
+
+
+def refresh_from_shards(W_shards, G_shards, M_shards, cfg: OracleConfig):
+    """Algorithm 2 lines 1-7 for one matrix, all ranks at once: every rank
+    updates the momentum of its rows, the rows are gathered into the full
+    momentum (here: concatenated), NS5 runs on the full matrix, and each rank
+    keeps its rows of the result.  Returns (new W shards, new M shards)."""
+    M_new = [momentum_update(M, G, cfg.beta) for M, G in zip(M_shards, G_shards)]
+    U_full = np.concatenate([direction_input(M, G, cfg.beta, cfg.nesterov) for M, G in zip(M_new, G_shards)], axis=0)
+    m, n = U_full.shape
+    D = shape_scale(m, n, cfg.scale_mode) * direction(U_full, True, cfg)
+    out, lo = [], 0
+    for W in W_shards:
+        hi = lo + W.shape[0]
+        out.append((1.0 - cfg.lr * cfg.wd) * W - cfg.lr * D[lo:hi])
+        lo = hi
+    return out, M_new

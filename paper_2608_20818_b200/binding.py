@@ -44,6 +44,7 @@ EXPORTS = (
     "prm_step_h2d", "prm_plan", "prm_status", "prm_last_error", "prm_launch_count", "prm_destroy",
     "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc", "prm_selftest_timeout", "prm_adamw_step",
     "prm_tall_shard_scratch_bytes", "prm_tall_shard_stats", "prm_tall_shard_apply", "prm_group_info",
+    "prm_shard_rows", "prm_bucket_plan", "prm_shard_momentum_pack", "prm_refresh_gathered", "prm_pipeline_model",
 )
 PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
 PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_GRAMSPACE, PRM_PROF_COUNT = 4, 5, 6, 7, 8
@@ -116,6 +117,19 @@ def lib():
     L.prm_tall_shard_apply.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int, c_float, c_int, c_float,
                                        c_float, c_float, c_float, c_float, c_void_p, c_void_p]
     L.prm_tall_shard_apply.restype = c_int
+    L.prm_shard_rows.argtypes = [c_int64, c_int, c_int, POINTER(c_int64), POINTER(c_int64)]
+    L.prm_shard_rows.restype = c_int
+    L.prm_bucket_plan.argtypes = [POINTER(c_int64), c_int, c_int, c_int64, POINTER(c_int), POINTER(c_int64),
+                                  POINTER(c_int), POINTER(c_int64)]
+    L.prm_bucket_plan.restype = c_int
+    L.prm_shard_momentum_pack.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int64, c_int, c_float, c_int,
+                                          c_void_p, c_void_p]
+    L.prm_shard_momentum_pack.restype = c_int
+    L.prm_refresh_gathered.argtypes = [c_void_p, POINTER(c_int), c_int, c_void_p, c_int64, POINTER(c_int64), c_int,
+                                       c_int, POINTER(c_void_p), c_void_p]
+    L.prm_refresh_gathered.restype = c_int
+    L.prm_pipeline_model.argtypes = [POINTER(c_double), POINTER(c_double), c_int, POINTER(c_double), POINTER(c_double)]
+    L.prm_pipeline_model.restype = c_int
     _lib_handle = L
     return L
 
@@ -242,6 +256,68 @@ def prm_adamw_step(params, grads, exp_avg, exp_avg_sq, step, *, lr=1e-4, beta1=0
                                     float(eps), float(wd), int(step), c_void_p(s))
     if code != PRM_OK:
         raise PrmError(code, "prm_adamw_step failed")
+
+
+def prm_shard_rows(rows, world, rank):
+    """(row_start, row_count) of one rank's dim-0 shard."""
+    start, count = c_int64(), c_int64()
+    code = lib().prm_shard_rows(int(rows), int(world), int(rank), byref(start), byref(count))
+    if code != PRM_OK:
+        raise PrmError(code, "prm_shard_rows: bad argument")
+    return start.value, count.value
+
+
+def prm_bucket_plan(shapes, world, bucket_bytes):
+    """(bucket_of_mat, offset_in_segment, segment_elems per bucket)."""
+    n = len(shapes)
+    flat = []
+    for (m, k) in shapes:
+        flat += [int(m), int(k)]
+    arr = (c_int64 * max(1, len(flat)))(*flat)
+    bucket = (c_int * max(1, n))()
+    off = (c_int64 * max(1, n))()
+    seg = (c_int64 * max(1, n))()
+    nb = c_int()
+    code = lib().prm_bucket_plan(arr, n, int(world), int(bucket_bytes), bucket, off, byref(nb), seg)
+    if code != PRM_OK:
+        raise PrmError(code, "prm_bucket_plan: bad argument")
+    return list(bucket)[:n], list(off)[:n], list(seg)[:nb.value]
+
+
+def prm_shard_momentum_pack(grad_shard, momentum_shard, cols, reserved_elems, beta, nesterov, u_out_ptr, stream=None):
+    """grad_shard, momentum_shard: (rows_local, cols) CUDA tensors (rows_local may be 0)."""
+    rows_local = int(grad_shard.shape[0])
+    s = stream if stream is not None else torch.cuda.current_stream(grad_shard.device).cuda_stream
+    with torch.cuda.device(grad_shard.device):
+        code = lib().prm_shard_momentum_pack(c_void_p(grad_shard.data_ptr()), c_void_p(momentum_shard.data_ptr()),
+                                             rows_local, int(cols), int(reserved_elems),
+                                             1 if grad_shard.dtype == torch.float32 else 0, float(beta),
+                                             int(bool(nesterov)), c_void_p(int(u_out_ptr)), c_void_p(s))
+    if code != PRM_OK:
+        raise PrmError(code, "prm_shard_momentum_pack failed")
+
+
+def prm_refresh_gathered(h, mats, gathered_ptr, segment_elems, offsets, world, rank, param_shard_ptrs, stream):
+    n = len(mats)
+    m = (c_int * max(1, n))(*[int(x) for x in mats])
+    o = (c_int64 * max(1, n))(*[int(x) for x in offsets])
+    p = (c_void_p * max(1, n))(*[c_void_p(int(x)) if x else None for x in param_shard_ptrs])
+    _check(lib().prm_refresh_gathered(h, m, n, c_void_p(int(gathered_ptr)), int(segment_elems), o, int(world),
+                                      int(rank), p, c_void_p(stream)), h)
+
+
+def prm_pipeline_model(a, c):
+    """(t_pipe, t_comm_exposed) of the ideal two-stage pipeline."""
+    n = len(a)
+    if n != len(c) or n < 1:
+        raise ValueError("a and c must have the same, positive length")
+    aa = (c_double * n)(*[float(x) for x in a])
+    cc = (c_double * n)(*[float(x) for x in c])
+    tp, te = c_double(), c_double()
+    code = lib().prm_pipeline_model(aa, cc, n, byref(tp), byref(te))
+    if code != PRM_OK:
+        raise PrmError(code, "prm_pipeline_model: bad argument")
+    return tp.value, te.value
 
 
 def prm_destroy(h):

@@ -260,127 +260,219 @@ extern "C" int prm_group_info(const prm_ctx* c, int group, int64_t* rows, int64_
   return PRM_OK;
 }
 
-static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepScalars s,
-                         cudaStream_t stream) {
+// Where the last NS5 iteration puts its result: straight into the parameters
+// (Eq. periodic-direction with rho_t = 1), or, with no NsFinal, into the
+// workspace as X_5.
+struct NsFinal {
+  PtrTables tables;
+  int first;          // table index of the sub-batch's first matrix
+  float decay, lr_s;
+};
+
+// The NS5 products of one sub-batch of nb matrices of group g whose oriented
+// input U already sits in the first X buffer of the NS5 region, alpha computed.
+// Returns the index (0 or 1) of the X buffer that holds X_5 when fin is null.
+static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFinal* fin, int* x_out,
+                                cudaStream_t stream) {
   const size_t e = c->check_mode ? 4 : 2;
   const int64_t rc = g.rp * g.cp, rr = g.rp * g.rp;
-  float* fro = (float*)(c->ws + c->off_fro);
   float* alpha = (float*)(c->ws + c->off_alpha);
   int* status = (int*)(c->ws + c->off_status);
+  char* base = c->ws + c->off_ns;
+  char* X[2] = {base, base + e * rc * nb};
+  char* R[4];                                      // r x r matrices (lower blocks)
+  for (int k = 0; k < 4; ++k) R[k] = base + 2 * e * rc * nb + (size_t)k * e * rr * nb;
+  char* A = R[0];
+  char* B = R[1];
+  cudaError_t ce;
+  auto gemm = [&](const GemmProblem& pb, const Epilogue& ep, int cls) -> cudaError_t {
+    ProfScope ps(c, cls, stream);
+    return c->check_mode ? launch_gemm_simt(pb, ep, stream, &c->launches)
+                         : launch_gemm_tc(c->tc, pb, ep, status, stream, &c->launches);
+  };
+  int cur = 0, it0 = 0;
+  ce = cudaSuccess;
+  if (g.gram_iters) {
+    // The first three iterations without touching X (tensor-core path).  With
+    // P_k = aI + B_k, B_k = bA_k + cA_k^2, the recurrence reads X_{k+1} = P_k X_k
+    // and A_{k+1} = X_{k+1} X_{k+1}^T = P_k A_k P_k, all polynomials in A_0 and
+    // therefore symmetric and commuting.  So A_1, A_2 follow from r x r products,
+    // and X_3 = (P_2 P_1 P_0) X_0 = a^3 X_0 + Q X_0 needs one r x c product, where
+    // Q (the product without its a^3 I term, which stays an fp32 coefficient) is
+    // accumulated beside.  In exact arithmetic this is the printed recurrence;
+    // the last two iterations, whose rounding decides the error, run as printed.
+    auto sym = [&](const char* Pm, const char* Qm, float k_acc, const char* aux, float k_aux, const char* aux2,
+                   float k_aux2, char* dst, int cls) -> cudaError_t {
+      GemmProblem pb;
+      pb.P = Pm; pb.Q = Qm; pb.Mp = g.rp; pb.Np = g.rp; pb.Kp = g.rp;
+      pb.bs_P = rr; pb.bs_Q = rr; pb.batch = nb; pb.symmetric = 1; pb.sym_ops = 3;
+      Epilogue ep;
+      ep.k_acc = k_acc; ep.k_aux = k_aux; ep.aux = aux; ep.ld_aux = g.rp; ep.bs_aux = rr;
+      if (aux2) { ep.aux2 = aux2; ep.k_aux2 = k_aux2; ep.ld_aux2 = g.rp; ep.bs_aux2 = rr; }
+      ep.dst = dst; ep.ld_dst = g.rp; ep.bs_dst = rr;
+      return gemm(pb, ep, cls);
+    };
+    auto poly = [&](const char* Am, char* Bm) { return sym(Am, Am, kNsC, Am, kNsB, nullptr, 0.f, Bm, PRM_PROF_POLY); };
+    const float a = kNsA;
+    GemmProblem pa;
+    pa.P = X[0]; pa.Q = X[0]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
+    pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
+    Epilogue ea;
+    ea.dst = R[0]; ea.ld_dst = g.rp; ea.bs_dst = rr; ea.alpha = alpha; ea.alpha_pow = 2;
+    ce = gemm(pa, ea, PRM_PROF_GRAM);                                                          // A_0
+    if (ce == cudaSuccess) ce = poly(R[0], R[1]);                                              // B_0
+    if (ce == cudaSuccess) ce = sym(R[0], R[1], 1.f, R[0], a, nullptr, 0.f, R[2], PRM_PROF_GRAMSPACE);   // Z = A_0 P_0
+    if (ce == cudaSuccess) ce = sym(R[2], R[1], 1.f, R[2], a, nullptr, 0.f, R[0], PRM_PROF_GRAMSPACE);   // A_1 = Z P_0
+    if (ce == cudaSuccess) ce = poly(R[0], R[3]);                                              // B_1
+    if (ce == cudaSuccess)                                                                     // Q = P_1 P_0 - a^2 I
+      ce = sym(R[3], R[1], 1.f, R[1], a, R[3], a, R[2], PRM_PROF_GRAMSPACE);
+    if (ce == cudaSuccess) ce = sym(R[0], R[3], 1.f, R[0], a, nullptr, 0.f, R[1], PRM_PROF_GRAMSPACE);   // Z = A_1 P_1
+    if (ce == cudaSuccess) ce = sym(R[1], R[3], 1.f, R[1], a, nullptr, 0.f, R[0], PRM_PROF_GRAMSPACE);   // A_2 = Z P_1
+    if (ce == cudaSuccess) ce = poly(R[0], R[3]);                                              // B_2
+    if (ce == cudaSuccess)                                                                     // Q = P_2 P_1 P_0 - a^3 I
+      ce = sym(R[3], R[2], 1.f, R[2], a, R[3], a * a, R[1], PRM_PROF_GRAMSPACE);
+    if (ce == cudaSuccess) {                                                                   // X_3 = alpha (a^3 X_0 + Q X_0)
+      GemmProblem pu;
+      pu.P = R[1]; pu.Q = X[0]; pu.q_mn = 1; pu.sym_ops = 1; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
+      pu.bs_P = rr; pu.bs_Q = rc; pu.batch = nb; pu.symmetric = 0;
+      Epilogue eu;
+      eu.k_acc = 1.f; eu.k_aux = a * a * a; eu.aux = X[0]; eu.ld_aux = g.cp; eu.bs_aux = rc;
+      eu.alpha = alpha; eu.alpha_pow = 1;
+      eu.dst = X[1]; eu.ld_dst = g.cp; eu.bs_dst = rc;
+      ce = gemm(pu, eu, PRM_PROF_UPDATE);
+    }
+    cur = 1;
+    it0 = kGramIters;
+  }
+  for (int it = it0; it < kNsIters && ce == cudaSuccess; ++it) {
+    // A = X X^T (times alpha^2 in the first iteration)
+    GemmProblem pa;
+    pa.P = X[cur]; pa.Q = X[cur]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
+    pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
+    Epilogue ea;
+    ea.dst = A; ea.ld_dst = g.rp; ea.bs_dst = rr;   // blocks on and below the diagonal only
+    if (it == 0) { ea.alpha = alpha; ea.alpha_pow = 2; }
+    if ((ce = gemm(pa, ea, PRM_PROF_GRAM)) != cudaSuccess) break;
+    // B = b A + c A^2
+    GemmProblem pp;
+    pp.P = A; pp.Q = A; pp.Mp = g.rp; pp.Np = g.rp; pp.Kp = g.rp;
+    pp.bs_P = rr; pp.bs_Q = rr; pp.batch = nb; pp.symmetric = 1; pp.sym_ops = 3;
+    Epilogue eb;
+    eb.k_acc = kNsC; eb.k_aux = kNsB; eb.aux = A; eb.ld_aux = g.rp; eb.bs_aux = rr;
+    eb.dst = B; eb.ld_dst = g.rp; eb.bs_dst = rr;
+    if ((ce = gemm(pp, eb, PRM_PROF_POLY)) != cudaSuccess) break;
+    // X <- a X + B X (times alpha in the first iteration); last iteration
+    // goes straight into the parameters.
+    GemmProblem pu;
+    // (B X)[i,j] = sum_k B[i,k] X[k,j]: X itself is the second operand, read with j contiguous.
+    pu.P = B; pu.Q = X[cur]; pu.q_mn = 1; pu.sym_ops = 1; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
+    pu.bs_P = rr; pu.bs_Q = rc; pu.batch = nb; pu.symmetric = 0;
+    Epilogue eu;
+    eu.k_acc = 1.f; eu.k_aux = kNsA; eu.aux = X[cur]; eu.ld_aux = g.cp; eu.bs_aux = rc;
+    if (it == 0) { eu.alpha = alpha; eu.alpha_pow = 1; }
+    if (it + 1 < kNsIters) {
+      eu.dst = X[cur ^ 1]; eu.ld_dst = g.cp; eu.bs_dst = rc;
+    } else if (!fin) {
+      eu.dst = X[cur ^ 1]; eu.ld_dst = g.cp; eu.bs_dst = rc;     // X_5 stays in the workspace
+    } else {
+      eu.kind = 1; eu.tables = fin->tables; eu.first = fin->first;
+      eu.rows = (int)g.rows; eu.cols = (int)g.cols; eu.tall = g.tall ? 1 : 0;
+      eu.io_fp32 = c->io_fp32; eu.decay = fin->decay; eu.lr_s = fin->lr_s;
+      // bf16 parameters with 16-byte aligned rows are updated through TMA-staged tiles.
+      if (!c->check_mode && !c->io_fp32 && g.cols % 8 == 0) eu.param_maps = c->ws + c->off_pmaps;
+    }
+    if ((ce = gemm(pu, eu, it + 1 < kNsIters ? PRM_PROF_UPDATE : PRM_PROF_UPDATE_FINAL)) != cudaSuccess) break;
+    cur ^= 1;
+  }
+  if (x_out) *x_out = cur;
+  return ce;
+}
+
+static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepScalars s,
+                         cudaStream_t stream) {
+  float* fro = (float*)(c->ws + c->off_fro);
+  float* alpha = (float*)(c->ws + c->off_alpha);
   for (int done = 0; done < g.count; done += g.ns_batch) {
     const int nb = std::min(g.ns_batch, g.count - done);
-    char* base = c->ws + c->off_ns;
-    char* X[2] = {base, base + e * rc * nb};
-    char* R[4];                                      // r x r matrices (lower blocks)
-    for (int k = 0; k < 4; ++k) R[k] = base + 2 * e * rc * nb + (size_t)k * e * rr * nb;
-    char* A = R[0];
-    char* B = R[1];
     const int first = g.first + done;
     cudaError_t ce;
     {
       ProfScope ps(c, PRM_PROF_PREPASS, stream);
-      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, c->check_mode, X[0], fro, alpha, stream,
+      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, c->check_mode, c->ws + c->off_ns, fro, alpha, stream,
                              &c->launches);
     }
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("pre-pass: ") + cudaGetErrorString(ce));
-    auto gemm = [&](const GemmProblem& pb, const Epilogue& ep, int cls) -> cudaError_t {
-      ProfScope ps(c, cls, stream);
-      return c->check_mode ? launch_gemm_simt(pb, ep, stream, &c->launches)
-                           : launch_gemm_tc(c->tc, pb, ep, status, stream, &c->launches);
-    };
-    int cur = 0, it0 = 0;
-    ce = cudaSuccess;
-    if (g.gram_iters) {
-      // The first three iterations without touching X (tensor-core path).  With
-      // P_k = aI + B_k, B_k = bA_k + cA_k^2, the recurrence reads X_{k+1} = P_k X_k
-      // and A_{k+1} = X_{k+1} X_{k+1}^T = P_k A_k P_k, all polynomials in A_0 and
-      // therefore symmetric and commuting.  So A_1, A_2 follow from r x r products,
-      // and X_3 = (P_2 P_1 P_0) X_0 = a^3 X_0 + Q X_0 needs one r x c product, where
-      // Q (the product without its a^3 I term, which stays an fp32 coefficient) is
-      // accumulated beside.  In exact arithmetic this is the printed recurrence;
-      // the last two iterations, whose rounding decides the error, run as printed.
-      auto sym = [&](const char* Pm, const char* Qm, float k_acc, const char* aux, float k_aux, const char* aux2,
-                     float k_aux2, char* dst, int cls) -> cudaError_t {
-        GemmProblem pb;
-        pb.P = Pm; pb.Q = Qm; pb.Mp = g.rp; pb.Np = g.rp; pb.Kp = g.rp;
-        pb.bs_P = rr; pb.bs_Q = rr; pb.batch = nb; pb.symmetric = 1; pb.sym_ops = 3;
-        Epilogue ep;
-        ep.k_acc = k_acc; ep.k_aux = k_aux; ep.aux = aux; ep.ld_aux = g.rp; ep.bs_aux = rr;
-        if (aux2) { ep.aux2 = aux2; ep.k_aux2 = k_aux2; ep.ld_aux2 = g.rp; ep.bs_aux2 = rr; }
-        ep.dst = dst; ep.ld_dst = g.rp; ep.bs_dst = rr;
-        return gemm(pb, ep, cls);
-      };
-      auto poly = [&](const char* Am, char* Bm) { return sym(Am, Am, kNsC, Am, kNsB, nullptr, 0.f, Bm, PRM_PROF_POLY); };
-      const float a = kNsA;
-      GemmProblem pa;
-      pa.P = X[0]; pa.Q = X[0]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
-      pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
-      Epilogue ea;
-      ea.dst = R[0]; ea.ld_dst = g.rp; ea.bs_dst = rr; ea.alpha = alpha; ea.alpha_pow = 2;
-      ce = gemm(pa, ea, PRM_PROF_GRAM);                                                          // A_0
-      if (ce == cudaSuccess) ce = poly(R[0], R[1]);                                              // B_0
-      if (ce == cudaSuccess) ce = sym(R[0], R[1], 1.f, R[0], a, nullptr, 0.f, R[2], PRM_PROF_GRAMSPACE);   // Z = A_0 P_0
-      if (ce == cudaSuccess) ce = sym(R[2], R[1], 1.f, R[2], a, nullptr, 0.f, R[0], PRM_PROF_GRAMSPACE);   // A_1 = Z P_0
-      if (ce == cudaSuccess) ce = poly(R[0], R[3]);                                              // B_1
-      if (ce == cudaSuccess)                                                                     // Q = P_1 P_0 - a^2 I
-        ce = sym(R[3], R[1], 1.f, R[1], a, R[3], a, R[2], PRM_PROF_GRAMSPACE);
-      if (ce == cudaSuccess) ce = sym(R[0], R[3], 1.f, R[0], a, nullptr, 0.f, R[1], PRM_PROF_GRAMSPACE);   // Z = A_1 P_1
-      if (ce == cudaSuccess) ce = sym(R[1], R[3], 1.f, R[1], a, nullptr, 0.f, R[0], PRM_PROF_GRAMSPACE);   // A_2 = Z P_1
-      if (ce == cudaSuccess) ce = poly(R[0], R[3]);                                              // B_2
-      if (ce == cudaSuccess)                                                                     // Q = P_2 P_1 P_0 - a^3 I
-        ce = sym(R[3], R[2], 1.f, R[2], a, R[3], a * a, R[1], PRM_PROF_GRAMSPACE);
-      if (ce == cudaSuccess) {                                                                   // X_3 = alpha (a^3 X_0 + Q X_0)
-        GemmProblem pu;
-        pu.P = R[1]; pu.Q = X[0]; pu.q_mn = 1; pu.sym_ops = 1; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
-        pu.bs_P = rr; pu.bs_Q = rc; pu.batch = nb; pu.symmetric = 0;
-        Epilogue eu;
-        eu.k_acc = 1.f; eu.k_aux = a * a * a; eu.aux = X[0]; eu.ld_aux = g.cp; eu.bs_aux = rc;
-        eu.alpha = alpha; eu.alpha_pow = 1;
-        eu.dst = X[1]; eu.ld_dst = g.cp; eu.bs_dst = rc;
-        ce = gemm(pu, eu, PRM_PROF_UPDATE);
-      }
-      cur = 1;
-      it0 = kGramIters;
-    }
-    for (int it = it0; it < kNsIters && ce == cudaSuccess; ++it) {
-      // A = X X^T (times alpha^2 in the first iteration)
-      GemmProblem pa;
-      pa.P = X[cur]; pa.Q = X[cur]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
-      pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
-      Epilogue ea;
-      ea.dst = A; ea.ld_dst = g.rp; ea.bs_dst = rr;   // blocks on and below the diagonal only
-      if (it == 0) { ea.alpha = alpha; ea.alpha_pow = 2; }
-      if ((ce = gemm(pa, ea, PRM_PROF_GRAM)) != cudaSuccess) break;
-      // B = b A + c A^2
-      GemmProblem pp;
-      pp.P = A; pp.Q = A; pp.Mp = g.rp; pp.Np = g.rp; pp.Kp = g.rp;
-      pp.bs_P = rr; pp.bs_Q = rr; pp.batch = nb; pp.symmetric = 1; pp.sym_ops = 3;
-      Epilogue eb;
-      eb.k_acc = kNsC; eb.k_aux = kNsB; eb.aux = A; eb.ld_aux = g.rp; eb.bs_aux = rr;
-      eb.dst = B; eb.ld_dst = g.rp; eb.bs_dst = rr;
-      if ((ce = gemm(pp, eb, PRM_PROF_POLY)) != cudaSuccess) break;
-      // X <- a X + B X (times alpha in the first iteration); last iteration
-      // goes straight into the parameters.
-      GemmProblem pu;
-      // (B X)[i,j] = sum_k B[i,k] X[k,j]: X itself is the second operand, read with j contiguous.
-      pu.P = B; pu.Q = X[cur]; pu.q_mn = 1; pu.sym_ops = 1; pu.Mp = g.rp; pu.Np = g.cp; pu.Kp = g.rp;
-      pu.bs_P = rr; pu.bs_Q = rc; pu.batch = nb; pu.symmetric = 0;
-      Epilogue eu;
-      eu.k_acc = 1.f; eu.k_aux = kNsA; eu.aux = X[cur]; eu.ld_aux = g.cp; eu.bs_aux = rc;
-      if (it == 0) { eu.alpha = alpha; eu.alpha_pow = 1; }
-      if (it + 1 < kNsIters) {
-        eu.dst = X[cur ^ 1]; eu.ld_dst = g.cp; eu.bs_dst = rc;
-      } else {
-        eu.kind = 1; eu.tables = t; eu.first = first;
-        eu.rows = (int)g.rows; eu.cols = (int)g.cols; eu.tall = g.tall ? 1 : 0;
-        eu.io_fp32 = c->io_fp32; eu.decay = s.decay; eu.lr_s = s.lr_s * c->gamma_ns;
-        // bf16 parameters with 16-byte aligned rows are updated through TMA-staged tiles.
-        if (!c->check_mode && !c->io_fp32 && g.cols % 8 == 0) eu.param_maps = c->ws + c->off_pmaps;
-      }
-      if ((ce = gemm(pu, eu, it + 1 < kNsIters ? PRM_PROF_UPDATE : PRM_PROF_UPDATE_FINAL)) != cudaSuccess) break;
-      cur ^= 1;
-    }
+    NsFinal fin{t, first, s.decay, s.lr_s * c->gamma_ns};
+    ce = ns5_products(c, g, nb, &fin, nullptr, stream);
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("NS5 product: ") + cudaGetErrorString(ce));
+  }
+  return PRM_OK;
+}
+
+// Refresh of a bucket of matrices whose rows arrived by all-gather
+// (Algorithm 2 lines 4-6 for one bucket, on one rank).
+extern "C" int prm_refresh_gathered(prm_ctx* c, const int* mats, int n, const void* gathered,
+                                    int64_t segment_elems, const int64_t* offsets, int world, int rank,
+                                    void* const* param_shards, void* cuda_stream) {
+  if (!c) return PRM_ERR_ARG;
+  if (!c->ws) return fail(c, PRM_ERR_WORKSPACE, "prm_refresh_gathered: no workspace attached");
+  if (n < 0 || (n > 0 && (!mats || !offsets || !param_shards || !gathered)))
+    return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: NULL argument");
+  if (world < 1 || rank < 0 || rank >= world) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: bad world or rank");
+  if (segment_elems < 0) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: negative segment size");
+  if (((uintptr_t)gathered & 15) != 0) return fail(c, PRM_ERR_ALIGN, "prm_refresh_gathered: buffer not 16-byte aligned");
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  for (int k = 0; k < n; ++k) {
+    if (mats[k] < 0 || mats[k] >= c->n_mats) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: matrix index out of range");
+    const Group& g = c->groups[c->group_of_mat[mats[k]]];
+    const int64_t chunk = shard_chunk(g.rows, world);
+    if (offsets[k] < 0 || offsets[k] + chunk * g.cols > segment_elems)
+      return fail(c, PRM_ERR_SHAPE, "prm_refresh_gathered: a matrix does not fit its segment");
+    int64_t start, count;
+    shard_rows(g.rows, world, rank, &start, &count);
+    if (count > 0) {
+      if (!param_shards[k]) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: NULL parameter shard");
+      if (((uintptr_t)param_shards[k] & (c->io_fp32 ? 3 : 1)) != 0)
+        return fail(c, PRM_ERR_ALIGN, "prm_refresh_gathered: parameter shard not aligned to its element size");
+    }
+  }
+  float* fro = (float*)(c->ws + c->off_fro);
+  float* alpha = (float*)(c->ws + c->off_alpha);
+  const size_t e = c->check_mode ? 4 : 2;
+  std::vector<int64_t> offs;
+  std::vector<void*> shards;
+  for (size_t gi = 0; gi < c->groups.size(); ++gi) {
+    const Group& g = c->groups[gi];
+    offs.clear();
+    shards.clear();
+    for (int k = 0; k < n; ++k)
+      if (c->group_of_mat[mats[k]] == (int)gi) { offs.push_back(offsets[k]); shards.push_back(param_shards[k]); }
+    if (offs.empty()) continue;
+    int64_t row_start, rows_local;
+    shard_rows(g.rows, world, rank, &row_start, &rows_local);
+    const float decay = 1.f - c->lr * c->wd;
+    const float lr_s = c->lr * shape_scale(c->scale_mode, g.rows, g.cols) * c->gamma_ns;
+    const int total = (int)offs.size();
+    for (int done = 0; done < total; done += g.ns_batch) {
+      const int nb = std::min(g.ns_batch, total - done);
+      cudaError_t ce;
+      {
+        ProfScope ps(c, PRM_PROF_PREPASS, stream);
+        ce = launch_ns_gather_prepass(gathered, segment_elems, shard_chunk(g.rows, world), offs.data() + done, g, nb,
+                                      c->eps_ns, c->check_mode, c->ws + c->off_ns, fro, alpha, stream, &c->launches);
+      }
+      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("gathered pre-pass: ") + cudaGetErrorString(ce));
+      int xi = 0;
+      ce = ns5_products(c, g, nb, nullptr, &xi, stream);
+      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("NS5 product: ") + cudaGetErrorString(ce));
+      {
+        ProfScope ps(c, PRM_PROF_UPDATE_FINAL, stream);
+        const char* X5 = c->ws + c->off_ns + (size_t)xi * e * (size_t)(g.rp * g.cp) * nb;
+        ce = launch_ns_slice_update(X5, c->check_mode, g, nb, shards.data() + done, row_start, rows_local, c->io_fp32,
+                                    decay, lr_s, stream, &c->launches);
+      }
+      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("slice update: ") + cudaGetErrorString(ce));
+    }
   }
   return PRM_OK;
 }

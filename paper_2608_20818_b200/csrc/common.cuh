@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <algorithm>
 #include <string>
 #include <vector>
 
@@ -114,6 +115,13 @@ __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ void from_f32(__nv_bfloat16* p, float x) { *p = __float2bfloat16_rn(x); }
 __device__ __forceinline__ void from_f32(float* p, float x) { *p = x; }
 
+// beta*x + omb*y in one fixed rounding order (a product, then a fused
+// multiply-add), so that every kernel that updates the momentum or forms the
+// direction input produces the same bits whatever else it does.
+__device__ __forceinline__ float blend(float beta, float x, float omb, float y) {
+  return __fmaf_rn(beta, x, __fmul_rn(omb, y));
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -154,5 +162,16 @@ struct Group {
 };
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+// dim-0 sharding as torch.chunk does it: rank q of `world` owns stored rows
+// [start, start + count) with chunk = ceil(rows / world).
+inline int64_t shard_chunk(int64_t rows, int world) { return (rows + world - 1) / world; }
+inline void shard_rows(int64_t rows, int world, int rank, int64_t* start, int64_t* count) {
+  const int64_t chunk = shard_chunk(rows, world);
+  const int64_t lo = std::min(rows, (int64_t)rank * chunk);
+  const int64_t hi = std::min(rows, lo + chunk);
+  *start = lo;
+  *count = hi - lo;
+}
 
 }  // namespace prm

@@ -73,6 +73,27 @@ cudaError_t launch_ns_prepass(const PtrTables& t, const Group& g, int first, int
                               float* fro_partial, float* alpha, cudaStream_t stream,
                               int64_t* launches);
 
+// alpha[b] = 1/(sqrt(sum of nparts partials of matrix b) + eps_ns).
+void launch_ns_alpha(const float* fro_partial, int nparts, float eps_ns, float* alpha, int batch,
+                     cudaStream_t stream);
+
+// Refresh over row shards (Algorithm 2 lines 1-7).  Matrices of one launch
+// are described by value, kGatherMax at a time.
+constexpr int kGatherMax = 32;
+struct GatherBatch { int64_t off[kGatherMax]; };   // element offset of the matrix inside every rank's segment
+struct SliceBatch { void* param[kGatherMax]; };    // this rank's parameter rows
+// The pre-pass on gathered rows: bf16 U of `batch` matrices of group g, read
+// from `world` segments of segment_elems elements (rank q at q*segment_elems),
+// row i of a matrix at segment i / chunk_rows, local row i % chunk_rows.
+cudaError_t launch_ns_gather_prepass(const void* gathered, int64_t segment_elems, int64_t chunk_rows,
+                                     const int64_t* offs, const Group& g, int batch, float eps_ns, int x_fp32,
+                                     void* X, float* fro_partial, float* alpha, cudaStream_t stream,
+                                     int64_t* launches);
+// W_shard <- decay*W_shard - lr_s*X5 on stored rows [row_start, row_start + rows_local).
+cudaError_t launch_ns_slice_update(const void* X5, int x_fp32, const Group& g, int batch,
+                                   void* const* param_shards, int64_t row_start, int64_t rows_local, int io_fp32,
+                                   float decay, float lr_s, cudaStream_t stream, int64_t* launches);
+
 // fp32 CUDA-core product (check mode).
 cudaError_t launch_gemm_simt(const GemmProblem& pb, const Epilogue& ep, cudaStream_t stream,
                              int64_t* launches);

@@ -50,9 +50,9 @@ ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
           load8_stream(m + off, mv);
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
-            const float mn = s.beta * mv[e] + s.omb * gv[e];
+            const float mn = blend(s.beta, mv[e], s.omb, gv[e]);
             mv[e] = mn;
-            u[e] = s.nesterov ? s.beta * mn + s.omb * gv[e] : mn;
+            u[e] = s.nesterov ? blend(s.beta, mn, s.omb, gv[e]) : mn;
           }
           store8(m + off, mv);
         }
@@ -61,9 +61,9 @@ ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
         for (int e = 0; e < 8; ++e) {
           if (col + e < cols) {
             const float gv = to_f32(g[off + e]);
-            const float mn = s.beta * m[off + e] + s.omb * gv;
+            const float mn = blend(s.beta, m[off + e], s.omb, gv);
             m[off + e] = mn;
-            u[e] = s.nesterov ? s.beta * mn + s.omb * gv : mn;
+            u[e] = s.nesterov ? blend(s.beta, mn, s.omb, gv) : mn;
           }
         }
       }
@@ -111,6 +111,11 @@ ns_alpha_kernel(const float* __restrict__ fro_partial, int nparts, float eps_ns,
     __syncthreads();
   }
   if (threadIdx.x == 0) alpha[blockIdx.x] = 1.f / (sqrtf(part[0]) + eps_ns);
+}
+
+void launch_ns_alpha(const float* fro_partial, int nparts, float eps_ns, float* alpha, int batch,
+                     cudaStream_t stream) {
+  ns_alpha_kernel<<<batch, kPreThreads, 0, stream>>>(fro_partial, nparts, eps_ns, alpha);
 }
 
 template <typename IO, typename XT_>

@@ -59,9 +59,9 @@ rowstep_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s) {
       if (PREP) pv[k].load_stream(p + 8 * v);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const float mn = s.beta * mv[e] + s.omb * gv[e];
+        const float mn = blend(s.beta, mv[e], s.omb, gv[e]);
         mv[e] = mn;
-        const float uu = s.nesterov ? s.beta * mn + s.omb * gv[e] : mn;
+        const float uu = s.nesterov ? blend(s.beta, mn, s.omb, gv[e]) : mn;
         u[k][e] = uu;
         acc += uu * uu;
       }
@@ -120,8 +120,8 @@ rowstep_wide_generic_kernel(PtrTables t, int first, int rows, int cols, StepScal
   float acc = 0.f;
   for (int j = threadIdx.x; j < cols; j += kRowThreads) {
     const float gv = to_f32(g[j]);
-    const float mn = s.beta * m[j] + s.omb * gv;
-    const float uu = s.nesterov ? s.beta * mn + s.omb * gv : mn;
+    const float mn = blend(s.beta, m[j], s.omb, gv);
+    const float uu = s.nesterov ? blend(s.beta, mn, s.omb, gv) : mn;
     acc += uu * uu;
   }
   acc = warp_sum(acc);
@@ -134,8 +134,8 @@ rowstep_wide_generic_kernel(PtrTables t, int first, int rows, int cols, StepScal
   const float coef = s.lr_s * s.gamma / nu;
   for (int j = threadIdx.x; j < cols; j += kRowThreads) {
     const float gv = to_f32(g[j]);
-    const float mn = s.beta * m[j] + s.omb * gv;
-    const float uu = s.nesterov ? s.beta * mn + s.omb * gv : mn;
+    const float mn = blend(s.beta, m[j], s.omb, gv);
+    const float uu = s.nesterov ? blend(s.beta, mn, s.omb, gv) : mn;
     m[j] = mn;
     from_f32(p + j, s.decay * to_f32(p[j]) - coef * uu);
   }
@@ -170,17 +170,17 @@ rowstep_tall_pass1_kernel(PtrTables t, int first, int rows, int cols, StepScalar
         load8(m + off, mv);
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-          const float mn = s.beta * mv[e] + s.omb * gv[e];
+          const float mn = blend(s.beta, mv[e], s.omb, gv[e]);
           mv[e] = mn;
-          const float uu = s.nesterov ? s.beta * mn + s.omb * gv[e] : mn;
+          const float uu = s.nesterov ? blend(s.beta, mn, s.omb, gv[e]) : mn;
           cs[e] += uu * uu;
         }
         store8(m + off, mv);
       } else {
         const float gv = to_f32(g[off]);
-        const float mn = s.beta * m[off] + s.omb * gv;
+        const float mn = blend(s.beta, m[off], s.omb, gv);
         m[off] = mn;
-        const float uu = s.nesterov ? s.beta * mn + s.omb * gv : mn;
+        const float uu = s.nesterov ? blend(s.beta, mn, s.omb, gv) : mn;
         cs[0] += uu * uu;
       }
     }
@@ -241,14 +241,14 @@ rowstep_tall_pass2_kernel(PtrTables t, int first, int rows, int cols, StepScalar
         float gv[8];
         load8_stream(g + off, gv);
 #pragma unroll
-        for (int e = 0; e < 8; ++e) mv[e] = s.beta * mv[e] + s.omb * gv[e];
+        for (int e = 0; e < 8; ++e) mv[e] = blend(s.beta, mv[e], s.omb, gv[e]);
       }
 #pragma unroll
       for (int e = 0; e < 8; ++e) pv[e] = s.decay * pv[e] - coef[e] * mv[e];
       store8(p + off, pv);
     } else {
       float uu = m[off];
-      if (s.nesterov) uu = s.beta * uu + s.omb * to_f32(g[off]);
+      if (s.nesterov) uu = blend(s.beta, uu, s.omb, to_f32(g[off]));
       from_f32(p + off, s.decay * to_f32(p[off]) - coef[0] * uu);
     }
   }

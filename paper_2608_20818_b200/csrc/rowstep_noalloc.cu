@@ -56,9 +56,9 @@ na_pass1_kernel(const IO* __restrict__ g, float* __restrict__ m, int rows, int c
       load8(m + off, mv);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        const float mn = beta * mv[e] + omb * gv[e];
+        const float mn = blend(beta, mv[e], omb, gv[e]);
         mv[e] = mn;
-        const float uu = nesterov ? beta * mn + omb * gv[e] : mn;
+        const float uu = nesterov ? blend(beta, mn, omb, gv[e]) : mn;
         cs[e] += uu * uu;
       }
       store8(m + off, mv);
@@ -109,7 +109,7 @@ na_pass2_kernel(IO* __restrict__ p, const IO* __restrict__ g, const float* __res
       float gv[8];
       load8_stream(g + off, gv);
 #pragma unroll
-      for (int e = 0; e < 8; ++e) mv[e] = beta * mv[e] + omb * gv[e];
+      for (int e = 0; e < 8; ++e) mv[e] = blend(beta, mv[e], omb, gv[e]);
     }
 #pragma unroll
     for (int e = 0; e < 8; ++e) pv[e] = decay * pv[e] - coef[e] * mv[e];

@@ -1,12 +1,20 @@
-"""Row step over dim-0 shards (the non-refresh branch of the paper's
-Algorithm 2): local column statistics of the tall matrices, one packed sum
-all-reduce, the wide matrices' row steps while it is in flight, then the tall
-matrices finished with the global norms.
+"""The paper's distributed execution (Section 3.3, Algorithm 2) over dim-0
+row shards, one process per GPU.
+
+Non-refresh branch (`sharded_row_step`): local column statistics of the tall
+matrices, one packed sum all-reduce, the wide matrices' row steps while it is
+in flight, then the tall matrices finished with the global norms.
+
+Refresh branch (`bucketed_refresh_step`): the Muon matrices travel in
+communication buckets; while the direction input of bucket l+1 is all-gathered,
+the matrices of bucket l are rebuilt, run through NS5 and sliced back to the
+local rows.
 
 Only orchestration lives here: the arithmetic runs in the CUDA library
-(`prm_tall_shard_stats`, `prm_tall_shard_apply`, `prm_step`), the exchange is
-`torch.distributed.all_reduce`.  The backend object is injectable so that the
-ordering and the packing can be exercised on CPU ranks.
+(`prm_tall_shard_stats`, `prm_tall_shard_apply`, `prm_step`,
+`prm_shard_momentum_pack`, `prm_refresh_gathered`), the exchanges are
+`torch.distributed` collectives (NCCL on GPUs).  The backend objects are
+injectable so that ordering, packing and slicing can be exercised on CPU ranks.
 """
 
 from __future__ import annotations
@@ -91,3 +99,120 @@ def sharded_row_step(tall, wide_step, backend, group=None, stream=0, stats_dtype
         cols = p.shape[1]
         backend.apply(p, g, m, packed[o:o + cols], math.sqrt(max(1.0, global_rows / cols)), stream)
     return packed
+
+
+# --------------------------------------------------------------------------
+# Refresh branch (Algorithm 2 lines 1-7): bucketed all-gather of the direction
+# input, NS5 on the rebuilt matrices while the next bucket is in flight,
+# results sliced back to the local rows.
+
+
+class CudaRefreshBackend:
+    """Marshals to prm_bucket_plan, prm_shard_momentum_pack and
+    prm_refresh_gathered.  `opt` is a PeriodicRowwiseMuon handle over the
+    GLOBAL shapes (its lr, wd, scale mode and NS5 options apply)."""
+
+    payload_dtype = torch.bfloat16
+
+    def __init__(self, opt, beta, nesterov):
+        self.opt = opt
+        self.beta = beta
+        self.nesterov = nesterov
+
+    def plan(self, shapes, world, bucket_bytes):
+        return B.prm_bucket_plan(shapes, world, bucket_bytes)
+
+    def shard_rows(self, rows, world, rank):
+        return B.prm_shard_rows(rows, world, rank)
+
+    def pack(self, grad, mom, cols, reserved, out, stream):
+        B.prm_shard_momentum_pack(grad, mom, cols, reserved, self.beta, self.nesterov, out.data_ptr(), stream)
+
+    def refresh(self, mats, gathered, segment_elems, offsets, world, rank, param_shards, stream):
+        ptrs = [p.data_ptr() if p.numel() else 0 for p in param_shards]
+        with torch.cuda.device(gathered.device):
+            B.prm_refresh_gathered(self.opt.h, mats, gathered.data_ptr(), segment_elems, offsets, world, rank, ptrs,
+                                   stream)
+
+
+def _all_gather(recv, send, group):
+    import torch.distributed as td
+    try:
+        return td.all_gather_into_tensor(recv, send, group=group, async_op=True)
+    except (RuntimeError, NotImplementedError):       # transports without the flat form
+        return td.all_gather(list(recv.chunk(td.get_world_size(group))), send, group=group, async_op=True)
+
+
+def bucketed_refresh_step(shapes, param_shards, grad_shards, mom_shards, backend, bucket_bytes=240 << 20,
+                          group=None, world=None, rank=None, buffers=None, trace=None):
+    """One refresh step over this rank's row shards (Algorithm 2 lines 1-7).
+
+    shapes        GLOBAL (rows, cols) of the Muon matrices, in the handle's order
+    *_shards      this rank's rows of every matrix (torch.chunk split of dim 0;
+                  a rank may own no row of a matrix: shape (0, cols))
+    backend       object with plan / shard_rows / pack / refresh and a
+                  payload_dtype (CudaRefreshBackend on GPUs)
+    bucket_bytes  cap on the gathered payload of one bucket
+    buffers       optional dict that keeps the two send and two receive
+                  buffers between calls
+    trace         optional list that receives ("gather", l) / ("refresh", l)
+                  in issue order
+    Work is issued on torch's current stream; the all-gather of bucket l+1 is
+    in flight while bucket l is refreshed.  Without an initialised process
+    group (or with world == 1) the exchange is a local copy.
+    """
+    import torch.distributed as td
+
+    dist_on = td.is_available() and td.is_initialized() and td.get_world_size(group) > 1
+    if world is None:
+        world = td.get_world_size(group) if dist_on else 1
+    if rank is None:
+        rank = td.get_rank(group) if dist_on else 0
+    if not dist_on and world != 1:
+        raise ValueError("world > 1 needs an initialised torch.distributed process group")
+    n = len(shapes)
+    bucket_of_mat, offsets, segments = backend.plan(shapes, world, bucket_bytes)
+    n_buckets = len(segments)
+    members = [[i for i in range(n) if bucket_of_mat[i] == l] for l in range(n_buckets)]
+    dev = param_shards[0].device
+    seg_max = max(segments)
+    if buffers is None:
+        buffers = {}
+    key = (seg_max, world, str(dev), backend.payload_dtype)
+    if buffers.get("key") != key:
+        buffers["key"] = key
+        buffers["send"] = [torch.empty(seg_max, dtype=backend.payload_dtype, device=dev) for _ in range(2)]
+        buffers["recv"] = [torch.empty(seg_max * world, dtype=backend.payload_dtype, device=dev) for _ in range(2)]
+    stream = torch.cuda.current_stream(dev).cuda_stream if dev.type == "cuda" else 0
+    pending = [None, None]
+
+    def launch(l):                                   # lines 2 and 4: pack, then gather asynchronously
+        send = buffers["send"][l % 2][:segments[l]]
+        recv = buffers["recv"][l % 2][:segments[l] * world]
+        for i in members[l]:
+            rows, cols = shapes[i]
+            chunk = -(-rows // world)
+            reserved = -(-(chunk * cols) // 8) * 8
+            backend.pack(grad_shards[i], mom_shards[i], cols, reserved, send[offsets[i]:offsets[i] + reserved], stream)
+        if trace is not None:
+            trace.append(("gather", l))
+        if dist_on:
+            pending[l % 2] = _all_gather(recv, send, group)
+        else:
+            recv.copy_(send)
+            pending[l % 2] = None
+
+    launch(0)
+    for l in range(n_buckets):
+        if pending[l % 2] is not None:               # line 4: wait for the current bucket ...
+            pending[l % 2].wait()
+            pending[l % 2] = None
+        if l + 1 < n_buckets:                        # ... and launch the next all-gather
+            launch(l + 1)
+        if trace is not None:
+            trace.append(("refresh", l))
+        recv = buffers["recv"][l % 2][:segments[l] * world]
+        backend.refresh(members[l], recv, segments[l], [offsets[i] for i in members[l]], world, rank,
+                        [param_shards[i] for i in members[l]], stream)      # line 5
+        # line 6: the buffers of bucket l are reused by bucket l + 2
+    return bucket_of_mat, offsets, segments

@@ -397,3 +397,24 @@ def test_refresh_gathered_rejects_bad_arguments():
     torch.cuda.synchronize()
     assert not p.any() and opt.status() == B.PRM_OK
     opt.close()
+
+
+@pytest.mark.gpu
+def test_bench_sharded_mode_single_rank_line():
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--sharded", "--config", "2", "--blocks", "2",
+                        "--K", "2", "--steps", "4", "--warmup", "3", "--bucket-mib", "64"], env=env,
+                       capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-800:]
+    line = json.loads(r.stdout.strip().splitlines()[-1])
+    assert line["scaling"] == "strong" and line["n_gpus"] == 1 and line["unit"] == "ms/step"
+    assert line["refresh_ms"] > line["row_step_ms"] > 0
+    pipe = line["pipeline"]
+    assert pipe["buckets"] == line["config"]["buckets"] >= 3
+    # the model's makespan lies between the compute alone and compute plus communication
+    assert pipe["compute_ms_sum"] <= pipe["t_pipe_model_ms"] <= pipe["compute_ms_sum"] + pipe["gather_ms_sum"] + 1e-6
+    assert pipe["gathered_payload_bytes"] == 2 * 2 * 18 * 2048 * 2048

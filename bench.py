@@ -140,11 +140,11 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------- CPU oracle
-def oracle_sample(wl, K, budget_s=20.0):
+def oracle_sample(wl, K, limit_s=20.0):
     """Times the fp64 oracle, as it stands, on a bounded sample of the workload
     and scales it to the whole shape set.  The sample is one matrix of each of
     the first distinct shapes of the set, as many as are predicted to fit the
-    time budget (always at least one; a square matrix smaller than d x d when
+    time limit (always at least one; a square matrix smaller than d x d when
     even that does not fit); each gets one refresh and one row step.  The
     refresh is scaled by the paper's flop model 20r^2c+10r^3, the row step by
     element count."""
@@ -180,12 +180,12 @@ def oracle_sample(wl, K, budget_s=20.0):
     rate = model(probe) / max(one(probe, 0), 1e-6)           # flop/s of the refresh at probe size
     sample, predicted = [], 0.0
     for sh in distinct:
-        if sample and predicted + model(sh) / rate > budget_s:
+        if sample and predicted + model(sh) / rate > limit_s:
             break
         sample.append(sh)
         predicted += model(sh) / rate
-    if len(sample) == 1 and model(sample[0]) / rate > budget_s:   # shrink the only matrix
-        r = max(64, int((budget_s * rate / 30.0) ** (1.0 / 3.0)) // 64 * 64)
+    if len(sample) == 1 and model(sample[0]) / rate > limit_s:   # shrink the only matrix
+        r = max(64, int((limit_s * rate / 30.0) ** (1.0 / 3.0)) // 64 * 64)
         sample = [(min(r, min(sample[0])),) * 2]
     t_ref = sum(one(sh, 0) for sh in sample)
     t_row = sum(one(sh, 1) for sh in sample) if K > 1 else 0.0
@@ -209,7 +209,7 @@ def run_reference(args, wl, K):
     base = None
     per = max(2.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
     for i in range(args.warmup + args.steps):
-        base = oracle_sample(wl, K, budget_s=per)
+        base = oracle_sample(wl, K, limit_s=per)
         if i >= args.warmup:
             vals.append(base["value"])
     v = sum(vals) / len(vals)

@@ -22,7 +22,7 @@ struct prm_ctx {
   int scale_mode = 1;
   int io_fp32 = 0;
   int check_mode = 0;
-  size_t ns_budget = (size_t)8 << 30;
+  size_t ns_cap = (size_t)8 << 30;
   float gamma_ns = 1.f;   // multiplier on the NS5 branch (ablation: "scalar-controlled" uses gamma)
   int no_refresh = 0;     // ablation: RowNorm at every step
   int gram_span = 1;      // first NS5 iterations in Gram space where it pays (tensor-core path)
@@ -118,7 +118,7 @@ static void compute_layout(prm_ctx* c) {
     g.gram_iters = (!c->check_mode && c->gram_span && g.rp >= 1024 && 2 * g.cp >= 3 * g.rp) ? kGramIters : 0;
     // X ping-pong, A, B (+ two more r x r matrices for the Gram-space iterations)
     const size_t per_mat = e * (size_t)(2 * g.rp * g.cp + (g.gram_iters ? 4 : 2) * g.rp * g.rp);
-    int nb = (int)std::min<size_t>((size_t)g.count, std::max<size_t>(1, c->ns_budget / per_mat));
+    int nb = (int)std::min<size_t>((size_t)g.count, std::max<size_t>(1, c->ns_cap / per_mat));
     // equal sub-batches: 42 matrices with room for 18 run as 14+14+14, not 18+18+6
     const int chunks = (g.count + nb - 1) / nb;
     nb = (g.count + chunks - 1) / chunks;
@@ -207,7 +207,7 @@ extern "C" int prm_set_option(prm_ctx* c, int key, double v) {
       if (attached) return fail(c, PRM_ERR_STATE, "option must be set before prm_set_workspace");
       if (key == PRM_OPT_NS_WORKSPACE_BYTES) {
         if (v < 0) return fail(c, PRM_ERR_ARG, "workspace cap must be >= 0");
-        c->ns_budget = (size_t)v;
+        c->ns_cap = (size_t)v;
       } else {
         if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
         (key == PRM_OPT_IO_DTYPE ? c->io_fp32 : key == PRM_OPT_CHECK_MODE ? c->check_mode : c->gram_span) = (int)v;

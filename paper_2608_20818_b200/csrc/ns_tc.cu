@@ -2,10 +2,12 @@
 // operands, fp32 accumulation in tensor memory, and the fused epilogues of
 // struct Epilogue (polynomial coefficients, Frobenius scale, final parameter
 // update).  Q may also be stored [k][n] (N-major operand), which is how the
-// update product reads X.  The symmetric matrices A and B exist only as their
-// 256x256 blocks on and below the diagonal: the products that consume them
-// read a missing block from its mirror image as an M/N-major operand, so no
-// product ever writes a transposed copy.
+// update product reads X.  The symmetric r x r matrices (A, B and, where the
+// first iterations run in Gram space, Z and the running product Q) exist only
+// as their 256x256 blocks on and below the diagonal: the products that consume
+// them read a missing block from its mirror image as an M/N-major operand, so
+// no product ever writes a transposed copy.  P and Q may be two different
+// symmetric matrices, and the epilogue takes up to two auxiliary operands.
 //
 // Persistent CTA pairs (clusters of two CTAs on two SMs), 352 threads per CTA.
 // A pair computes a 256x256 tile with tcgen05.mma.cta_group::2: each CTA holds

@@ -351,6 +351,21 @@ PRM_API int prm_refresh_gathered(prm_ctx* ctx, const int* mats, int n, const voi
 PRM_API int prm_pipeline_model(const double* a, const double* c, int n_buckets, double* t_pipe,
                                double* t_comm_exposed);
 
+/*
+ * The partition that needs no optimizer collective: whole matrices assigned
+ * to ranks.  Every matrix's update is independent of every other's (Algorithm
+ * 1 lines 4-10), so a rank that owns a matrix (parameter, gradient, momentum)
+ * runs prm_step on its own list and nothing is exchanged; Section 3.3's
+ * collectives exist only because dim-0 sharding splits each matrix.  Host
+ * only: longest-processing-time greedy on the NS5 cost 15 r^2 c + 5 r^3 of
+ * each matrix (decreasing cost, ties by index; least-loaded rank, ties by
+ * rank).  owner_of_mat[n_mats] receives the rank of each matrix, cost_out[world]
+ * (may be NULL) the flop assigned to each rank.  The paper does not describe
+ * this layout; it is offered beside the paper's.
+ */
+PRM_API int prm_partition_matrices(const int64_t* shapes, int n_mats, int world, int* owner_of_mat,
+                                   double* cost_out);
+
 /* Frees host resources.  Device memory belongs to the caller. */
 PRM_API int prm_destroy(prm_ctx* ctx);
 

@@ -45,6 +45,7 @@ EXPORTS = (
     "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc", "prm_selftest_timeout", "prm_adamw_step",
     "prm_tall_shard_scratch_bytes", "prm_tall_shard_stats", "prm_tall_shard_apply", "prm_group_info",
     "prm_shard_rows", "prm_bucket_plan", "prm_shard_momentum_pack", "prm_refresh_gathered", "prm_pipeline_model",
+    "prm_partition_matrices",
 )
 PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
 PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_GRAMSPACE, PRM_PROF_COUNT = 4, 5, 6, 7, 8
@@ -130,6 +131,8 @@ def lib():
     L.prm_refresh_gathered.restype = c_int
     L.prm_pipeline_model.argtypes = [POINTER(c_double), POINTER(c_double), c_int, POINTER(c_double), POINTER(c_double)]
     L.prm_pipeline_model.restype = c_int
+    L.prm_partition_matrices.argtypes = [POINTER(c_int64), c_int, c_int, POINTER(c_int), POINTER(c_double)]
+    L.prm_partition_matrices.restype = c_int
     _lib_handle = L
     return L
 
@@ -318,6 +321,21 @@ def prm_pipeline_model(a, c):
     if code != PRM_OK:
         raise PrmError(code, "prm_pipeline_model: bad argument")
     return tp.value, te.value
+
+
+def prm_partition_matrices(shapes, world):
+    """(owner_of_mat, flop per rank): whole matrices assigned to ranks."""
+    n = len(shapes)
+    flat = []
+    for (m, k) in shapes:
+        flat += [int(m), int(k)]
+    arr = (c_int64 * max(1, len(flat)))(*flat)
+    owner = (c_int * max(1, n))()
+    cost = (c_double * max(1, int(world)))()
+    code = lib().prm_partition_matrices(arr, n, int(world), owner, cost)
+    if code != PRM_OK:
+        raise PrmError(code, "prm_partition_matrices: bad argument")
+    return list(owner)[:n], list(cost)[:int(world)]
 
 
 def prm_destroy(h):

@@ -54,3 +54,35 @@ extern "C" int prm_pipeline_model(const double* a, const double* c, int n_bucket
   if (t_comm_exposed) *t_comm_exposed = exposed;
   return PRM_OK;
 }
+
+// Whole matrices assigned to ranks (no optimizer collective at all: every
+// matrix's update is independent of every other's, Algorithm 1 lines 4-10).
+// Longest-processing-time greedy on the refresh cost: matrices in decreasing
+// order of their executed NS5 flop (ties: lower index first) go to the rank
+// with the least load so far (ties: lower rank).  cost_out[q] receives the
+// load of rank q in flop (may be NULL).
+extern "C" int prm_partition_matrices(const int64_t* shapes, int n_mats, int world, int* owner_of_mat,
+                                      double* cost_out) {
+  if (!shapes || n_mats < 1 || world < 1 || !owner_of_mat) return PRM_ERR_ARG;
+  std::vector<double> cost(n_mats);
+  std::vector<int> order(n_mats);
+  for (int i = 0; i < n_mats; ++i) {
+    const int64_t m = shapes[2 * i], n = shapes[2 * i + 1];
+    if (m < 1 || n < 1) return PRM_ERR_SHAPE;
+    const double r = (double)std::min(m, n), c = (double)std::max(m, n);
+    cost[i] = 15.0 * r * r * c + 5.0 * r * r * r;      // printed recurrence with symmetric products
+    order[i] = i;
+  }
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cost[a] > cost[b]; });
+  std::vector<double> load(world, 0.0);
+  for (int k = 0; k < n_mats; ++k) {
+    int best = 0;
+    for (int q = 1; q < world; ++q)
+      if (load[q] < load[best]) best = q;
+    owner_of_mat[order[k]] = best;
+    load[best] += cost[order[k]];
+  }
+  if (cost_out)
+    for (int q = 0; q < world; ++q) cost_out[q] = load[q];
+  return PRM_OK;
+}

@@ -418,3 +418,27 @@ def test_bench_sharded_mode_single_rank_line():
     # the model's makespan lies between the compute alone and compute plus communication
     assert pipe["compute_ms_sum"] <= pipe["t_pipe_model_ms"] <= pipe["compute_ms_sum"] + pipe["gather_ms_sum"] + 1e-6
     assert pipe["gathered_payload_bytes"] == 2 * 2 * 18 * 2048 * 2048
+
+
+def test_partition_matrices_is_balanced_and_deterministic():
+    for cfg_id, world in ((4, 8), (2, 3), (3, 5), (5, 7)):
+        shapes = [tuple(s) for s in workload(cfg_id).shapes]
+        owner, load = B.prm_partition_matrices(shapes, world)
+        assert len(owner) == len(shapes) and set(owner) == set(range(world))
+        cost = [15 * min(s) ** 2 * max(s) + 5 * min(s) ** 3 for s in shapes]
+        for q in range(world):
+            assert load[q] == pytest.approx(sum(c for c, o in zip(cost, owner) if o == q), rel=1e-12)
+        # greedy longest-processing-time: no rank exceeds the mean by more than the largest matrix
+        assert max(load) <= sum(cost) / world + max(cost)
+        assert max(load) / (sum(cost) / world) < 1.1
+        assert B.prm_partition_matrices(shapes, world)[0] == owner
+    # brute force on a tiny case: the greedy result is within the list-scheduling bound of the optimum
+    shapes = [(8, 8), (8, 16), (8, 24), (8, 8), (8, 32)]
+    owner, load = B.prm_partition_matrices(shapes, 2)
+    cost = [15 * 64 * c + 5 * 512 for (_, c) in shapes]
+    best = min(max(sum(c for c, bit in zip(cost, range(5)) if (mask >> bit) & 1),
+                   sum(c for c, bit in zip(cost, range(5)) if not (mask >> bit) & 1)) for mask in range(32))
+    assert best <= max(load) <= (4 / 3 - 1 / 6) * best
+    assert B.prm_partition_matrices([(4, 4)], 3)[0] == [0]
+    with pytest.raises(B.PrmError):
+        B.prm_partition_matrices([(4, 4)], 0)

@@ -41,16 +41,17 @@ ROW_DRAM_BYTES_PER_ELEMENT = 14.0   # wide; the captures never exceed the algori
 
 
 # ----------------------------------------------------------------- accounting
-def ns5_flops(shapes, gram_iters=None):
-    """(executed, paper model) flop of one refresh.  Executed: the printed
-    recurrence with triangle-only symmetric products, 15r^2c+5r^3 per matrix, or
-    9r^2c+11r^3 where the library runs the first three iterations in Gram space
-    (gram_iters: {shape: 0 or 3}, as prm_group_info reports)."""
+def ns5_flops(shapes, exec_flop=None):
+    """(executed, paper model) flop of one refresh.  Executed: what the library
+    reports per matrix of each shape (exec_flop: {shape: flop}, from
+    prm_group_info: 9r^2c+11r^3 or 8r^2c+13r^3 where the first iterations run in
+    Gram space), else the printed recurrence with triangle-only symmetric
+    products, 15r^2c+5r^3."""
     ex = mo = 0
     for (m, n) in shapes:
         r, c = min(m, n), max(m, n)
-        if gram_iters and gram_iters.get((m, n), 0):
-            ex += 9 * r * r * c + 11 * r ** 3
+        if exec_flop and (m, n) in exec_flop:
+            ex += exec_flop[(m, n)]
         else:
             ex += 15 * r * r * c + 5 * r ** 3
         mo += 20 * r * r * c + 10 * r ** 3
@@ -405,6 +406,7 @@ def main():
                                 io_dtype=wl.io_dtype, check_mode=args.check_mode, gram_span=not args.printed_ns5,
                                 device=dev)
     gram_iters = {(g["rows"], g["cols"]): g["gram_iters"] for g in opt.groups()}
+    exec_flop = {(g["rows"], g["cols"]): g["ns5_flop"] for g in opt.groups()}
     params = [make_param(wl, i, dev) for i in range(n)]
     moms = [make_momentum(wl, i, dev) for i in range(n)]
     # One gradient set per matrix kind and step parity keeps generation cheap;
@@ -493,7 +495,7 @@ def main():
     pk = peaks()
     amort = (mean_ref + (K - 1) * mean_row) / K if (ref_ms and (row_ms or K == 1)) else total_ms / args.steps
     n_ref, n_row = len(ref_ms), len(row_ms)
-    ex, mo = ns5_flops(wl.shapes, gram_iters)
+    ex, mo = ns5_flops(wl.shapes, exec_flop)
     ex_printed, _ = ns5_flops(wl.shapes)
     el = elements(wl.shapes)
     row_bytes = el * (3 * io_bytes + 8)   # g and p read, p write (I/O dtype), m read and write (fp32)

@@ -76,8 +76,10 @@ extern "C" {
  * three iterations work on r x r matrices only (A_1, A_2 and the product of the
  * three factors aI + B_k from r x r products), then X_3 comes from one r x c
  * product and the last two iterations run as printed: 9 r^2 c + 11 r^3 flop
- * instead of 15 r^2 c + 5 r^3, the same result in exact arithmetic.  0: all five
- * iterations as printed.  The check mode always runs them as printed.  Before
+ * instead of 15 r^2 c + 5 r^3, the same result in exact arithmetic.  Beyond
+ * c = 2 r the Gram matrix of the fifth iteration is taken from the fourth's as
+ * well (A_4 = (aI + B_3) A_3 (aI + B_3), two r x r products instead of
+ * X_4 X_4^T): 8 r^2 c + 13 r^3.  0: all five iterations as printed.  The check mode always runs them as printed.  Before
  * set_workspace (the workspace holds two more r x r matrices per refreshed
  * matrix when this is on). */
 #define PRM_OPT_NS_GRAM_SPAN 12
@@ -151,12 +153,15 @@ PRM_API int prm_plan(const prm_ctx* ctx, int64_t step_idx, int* is_refresh,
 /*
  * One shape group of the plan (0 <= group < n_groups): its stored shape, the
  * number of matrices, how many of them one refresh sub-batch holds with the
- * current workspace cap, and how many leading NS5 iterations the refresh runs
- * in Gram space (0 or 3, see PRM_OPT_NS_GRAM_SPAN).  Host only.  Any output
- * pointer may be NULL.  PRM_ERR_ARG for a group out of range.
+ * current workspace cap, how many leading NS5 iterations the refresh runs in
+ * Gram space (0 or 3, see PRM_OPT_NS_GRAM_SPAN), and the flop one refresh of
+ * one such matrix executes in its NS5 products (X X^T products counted r^2 c,
+ * r x c products 2 r^2 c, symmetric r x r products r^3, r <= c the oriented
+ * shape).  Host only.  Any output pointer may be NULL.  PRM_ERR_ARG for a
+ * group out of range.
  */
 PRM_API int prm_group_info(const prm_ctx* ctx, int group, int64_t* rows, int64_t* cols,
-                   int* count, int* ns_batch, int* gram_iters);
+                   int* count, int* ns_batch, int* gram_iters, double* ns5_flop);
 
 /* Reads the device status word (synchronises the device first): PRM_OK, or
  * PRM_ERR_DEVICE_TIMEOUT if a kernel gave up on a bounded wait since the last

@@ -86,7 +86,7 @@ def lib():
     L.prm_plan.argtypes = [c_void_p, c_int64, POINTER(c_int), POINTER(c_int), POINTER(c_int), POINTER(c_int)]
     L.prm_plan.restype = c_int
     L.prm_group_info.argtypes = [c_void_p, c_int, POINTER(c_int64), POINTER(c_int64), POINTER(c_int), POINTER(c_int),
-                                 POINTER(c_int)]
+                                 POINTER(c_int), POINTER(c_double)]
     L.prm_group_info.restype = c_int
     L.prm_status.argtypes = [c_void_p]
     L.prm_status.restype = c_int
@@ -187,13 +187,14 @@ def prm_plan(h, step_idx, n_mats):
 
 
 def prm_group_info(h, group):
-    """{rows, cols, count, ns_batch, gram_iters} of one shape group."""
+    """{rows, cols, count, ns_batch, gram_iters, ns5_flop} of one shape group."""
     rows, cols = c_int64(), c_int64()
     count, ns_batch, gram_iters = c_int(), c_int(), c_int()
+    flop = c_double()
     _check(lib().prm_group_info(h, int(group), byref(rows), byref(cols), byref(count), byref(ns_batch),
-                                byref(gram_iters)), h)
+                                byref(gram_iters), byref(flop)), h)
     return {"rows": rows.value, "cols": cols.value, "count": count.value, "ns_batch": ns_batch.value,
-            "gram_iters": gram_iters.value}
+            "gram_iters": gram_iters.value, "ns5_flop": flop.value}
 
 
 def prm_status(h):

@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 
 TOL = 2e-2
 # (shape, Gram-space iterations expected): oriented rows padded to >= 1024 and padded c >= 1.5 r
-CASES = [((1024, 2048), 3), ((2048, 1024), 3), ((1100, 3000), 3), ((1024, 1536), 3), ((1280, 1792), 0),
+CASES = [((1024, 3072), 3), ((4096, 1024), 3), ((1024, 2048), 3), ((2048, 1024), 3), ((1100, 3000), 3), ((1024, 1536), 3), ((1280, 1792), 0),
          ((1024, 1024), 0), ((768, 3072), 0), ((1030, 2000), 3), ((3000, 1100), 3)]
 
 
@@ -39,15 +39,20 @@ def test_gramspace_direction_within_bound_and_eligibility(shape, iters):
 
 
 def test_gramspace_launch_classes_and_sub_batches():
-    shapes = [(1024, 2048)] * 3 + [(2048, 1024)] * 2 + [(512, 1024)]
+    # (1024, 2560): c > 2r, so the last Gram matrix comes from the one before it as well
+    shapes = [(1024, 2048)] * 3 + [(2048, 1024)] * 2 + [(512, 1024)] + [(1024, 2560)]
     cfg = U.oracle_cfg(K=1, nesterov=True, lr=1.0, wd=0.0, scale_mode=0)
     W, G, M = U.make_inputs(shapes, 17, "bf16", grad_std=1e-3, mom_std=1e-3)
     for w in W:
         w.zero_()
-    for ns_ws, sub_batches in ((None, (1, 1, 1)), (1, (3, 2, 1))):
+    for ns_ws, sub_batches in ((None, (1, 1, 1, 1)), (1, (3, 2, 1, 1))):
         opt = B.PeriodicRowwiseMuon(shapes, 1, 0.95, True, 1.0, 0.0, scale_mode=0, ns_workspace_bytes=ns_ws)
         info = opt.groups()
-        assert [g["gram_iters"] for g in info] == [3, 3, 0]
+        assert [g["gram_iters"] for g in info] == [3, 3, 0, 3]
+        r, c = 1024.0, 2560.0
+        assert info[3]["ns5_flop"] == 8 * r * r * c + 13 * r ** 3
+        assert info[0]["ns5_flop"] == 9 * r * r * 2048 + 11 * r ** 3
+        assert info[2]["ns5_flop"] == 15 * 512.0 ** 2 * 1024 + 5 * 512.0 ** 3
         w = [x.cuda() for x in W]
         g = [x.cuda() for x in G]
         m = [x.cuda() for x in M]
@@ -58,11 +63,12 @@ def test_gramspace_launch_classes_and_sub_batches():
         assert opt.status() == B.PRM_OK
         n_gram = sub_batches[0] + sub_batches[1]          # sub-batches refreshed in Gram space
         n_printed = sub_batches[2]
-        assert prof["gramspace"][1] == 6 * n_gram
-        assert prof["gram"][1] == 3 * n_gram + 5 * n_printed
-        assert prof["poly"][1] == 5 * (n_gram + n_printed)
-        assert prof["update"][1] == 2 * n_gram + 4 * n_printed
-        assert prof["update_final"][1] == n_gram + n_printed
+        n_rec = sub_batches[3]                            # ... and with the last Gram matrix by recurrence
+        assert prof["gramspace"][1] == 6 * n_gram + 8 * n_rec
+        assert prof["gram"][1] == 3 * n_gram + 5 * n_printed + 2 * n_rec
+        assert prof["poly"][1] == 5 * (n_gram + n_printed + n_rec)
+        assert prof["update"][1] == 2 * (n_gram + n_rec) + 4 * n_printed
+        assert prof["update_final"][1] == n_gram + n_printed + n_rec
         for i, s in enumerate(shapes):
             Wr, _ = O.step_matrix(U.to_np64(W[i]), U.to_np64(G[i]), U.to_np64(M[i]), 0, cfg)
             assert U.rel_fro(U.to_np64(w[i]), Wr) <= TOL, (i, s)

@@ -44,8 +44,7 @@ ROW_DRAM_BYTES_PER_ELEMENT = 14.0   # wide; the captures never exceed the algori
 def ns5_flops(shapes, exec_flop=None):
     """(executed, paper model) flop of one refresh.  Executed: what the library
     reports per matrix of each shape (exec_flop: {shape: flop}, from
-    prm_group_info: 9r^2c+11r^3 or 8r^2c+13r^3 where the first iterations run in
-    Gram space), else the printed recurrence with triangle-only symmetric
+    prm_group_info: 9r^2c+11r^3 where the first iterations run in Gram space), else the printed recurrence with triangle-only symmetric
     products, 15r^2c+5r^3."""
     ex = mo = 0
     for (m, n) in shapes:

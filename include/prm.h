@@ -76,10 +76,8 @@ extern "C" {
  * three iterations work on r x r matrices only (A_1, A_2 and the product of the
  * three factors aI + B_k from r x r products), then X_3 comes from one r x c
  * product and the last two iterations run as printed: 9 r^2 c + 11 r^3 flop
- * instead of 15 r^2 c + 5 r^3, the same result in exact arithmetic.  Beyond
- * c = 2 r the Gram matrix of the fifth iteration is taken from the fourth's as
- * well (A_4 = (aI + B_3) A_3 (aI + B_3), two r x r products instead of
- * X_4 X_4^T): 8 r^2 c + 13 r^3.  0: all five iterations as printed.  The check mode always runs them as printed.  Before
+ * instead of 15 r^2 c + 5 r^3, the same result in exact arithmetic.  0: all five
+ * iterations as printed.  The check mode always runs them as printed.  Before
  * set_workspace (the workspace holds two more r x r matrices per refreshed
  * matrix when this is on). */
 #define PRM_OPT_NS_GRAM_SPAN 12

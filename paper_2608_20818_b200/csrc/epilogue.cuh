@@ -11,7 +11,7 @@ namespace prm {
 // aux_prefetch); when null the auxiliary operand is loaded here.
 template <typename XT_, int N>
 __device__ __forceinline__ void epilogue_row(const Epilogue& ep, int b, int i, int j0,
-                                             float (&acc)[N], bool mirror, const float* pre = nullptr) {
+                                             float (&acc)[N], const float* pre = nullptr) {
   const float al = ep.alpha ? ep.alpha[b] : 1.f;
   const float f = ep.alpha_pow == 2 ? al * al : (ep.alpha_pow == 1 ? al : 1.f);
   const float ka = f * ep.k_acc, kx = f * ep.k_aux;
@@ -42,11 +42,6 @@ __device__ __forceinline__ void epilogue_row(const Epilogue& ep, int b, int i, i
 #pragma unroll
       for (int e = 0; e < 8; ++e) x[e] = acc[v + e];
       store8(dst + v, x);
-    }
-    if (mirror && ep.dst_t != nullptr) {
-      XT_* dt = reinterpret_cast<XT_*>(ep.dst_t) + (int64_t)b * ep.bs_dst_t + i;
-#pragma unroll
-      for (int e = 0; e < N; ++e) from_f32(dt + (int64_t)(j0 + e) * ep.ld_dst_t, acc[e]);
     }
   } else {
     // Parameter update at the stored position of oriented element (i, j).

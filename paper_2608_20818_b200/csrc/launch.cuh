@@ -10,10 +10,9 @@ namespace prm {
 // v = f*(k_acc*D[i,j] + k_aux*aux[i,j]):
 // (plus f*k_aux2*aux2[i,j] where a second auxiliary operand is given: the
 // Gram-space products of the tensor-core path)
-//   kind 0: dst[i,j] = v; if dst_t is set, dst_t[j,i] = v as well.  The
-//           symmetric products store only the blocks they compute (on and
-//           below the diagonal); their consumers read the mirrored block
-//           instead of the missing one (GemmProblem::sym_ops).
+//   kind 0: dst[i,j] = v.  The symmetric products store only the blocks they
+//           compute (on and below the diagonal); their consumers read the
+//           mirrored block instead of the missing one (GemmProblem::sym_ops).
 //   kind 1: parameter update W = decay*W - lr_s*v at the stored position of
 //           oriented element (i,j) (Eq. periodic-direction, rho_t = 1).
 struct Epilogue {
@@ -28,8 +27,6 @@ struct Epilogue {
   int64_t ld_aux2 = 0, bs_aux2 = 0;
   void* dst = nullptr;            // [batch][Mp][ld_dst]
   int64_t ld_dst = 0, bs_dst = 0;
-  void* dst_t = nullptr;          // [batch][Np][ld_dst_t]
-  int64_t ld_dst_t = 0, bs_dst_t = 0;
   // kind 1
   PtrTables tables = {};
   int first = 0;                  // table index of the sub-batch's first matrix

@@ -97,12 +97,11 @@ gemm_simt_kernel(GemmProblem pb, Epilogue ep) {
 #pragma unroll
     for (int c = 0; c < 8; ++c) tot[a][c] += acc[a][c];
 
-  const bool mirror = pb.symmetric ? (ti != tj) : true;
 #pragma unroll
   for (int a = 0; a < 8; ++a) {
     const int i = ti * kSimtTile + ty * 8 + a;
     const int j0 = tj * kSimtTile + tx * 8;
-    epilogue_row<float, 8>(ep, b, i, j0, tot[a], mirror);
+    epilogue_row<float, 8>(ep, b, i, j0, tot[a]);
   }
 }
 

@@ -60,7 +60,7 @@ constexpr int kSlabCols = 64;        // epilogue slab: 128 rows x 64 columns
 constexpr int kSlabs = 4;            // slabs per tile (kBN / kSlabCols)
 constexpr int kEpiBufs = 3;
 constexpr uint32_t kSlabBytes = 128 * kSlabCols * 2;        // result slab, also the aux slab
-constexpr uint32_t kEpiBufBytes = 2 * kSlabBytes;           // + transposed slab (2 boxes of 64x64)
+constexpr uint32_t kEpiBufBytes = 2 * kSlabBytes;           // + parameter tile or second auxiliary slab
 constexpr uint32_t kBytesA = kBM * kBK * 2;
 constexpr uint32_t kBytesB = (kBN / 2) * kBK * 2;   // each CTA of the pair holds half of Q's rows
 constexpr uint32_t kStageBytes = kBytesA + kBytesB;
@@ -222,7 +222,6 @@ __device__ __forceinline__ void tmem_ld_wait() {
 
 struct TileCoord {
   int b, ti, tj;
-  bool mirror;
 };
 __device__ __forceinline__ TileCoord decode_tile(int t, int tiles_per_mat, int symmetric, int mt) {
   TileCoord c;
@@ -233,11 +232,9 @@ __device__ __forceinline__ TileCoord decode_tile(int t, int tiles_per_mat, int s
     tri_decode(rem >> 1, bi, bj);      // 256x256 blocks of the lower triangle
     c.ti = 2 * bi + (rem & 1);         // two 128-row tiles per block
     c.tj = bj;
-    c.mirror = bi != bj;
   } else {
     c.ti = rem % mt;                   // row tiles fastest: concurrent CTAs share the Q panel
     c.tj = rem / mt;
-    c.mirror = true;
   }
   return c;
 }
@@ -249,14 +246,14 @@ template <int Q_MN, int SYM_OPS, int AUX2>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ,
                const __grid_constant__ CUtensorMap mapAux, const __grid_constant__ CUtensorMap mapAux2,
-               const __grid_constant__ CUtensorMap mapDst, const __grid_constant__ CUtensorMap mapDstT,
+               const __grid_constant__ CUtensorMap mapDst,
                const __grid_constant__ CUtensorMap mapSymP, const __grid_constant__ CUtensorMap mapSymQ,
                int ktiles, int tiles_per_mat, int total_tiles, int symmetric, int mt, Epilogue ep,
                int* status) {
   constexpr int q_mn = Q_MN, sym_ops = SYM_OPS;
   // AUX2: a second auxiliary operand (Epilogue::aux2) travels in the half of
-  // the slab buffer that the transposed result or the parameter tile would
-  // use; only the Gram-space products of two symmetric matrices need it.
+  // the slab buffer that the parameter tile of the final update uses; only the
+  // Gram-space products of two symmetric matrices need it.
   // q_mn: Q is stored [k][n] (n contiguous) instead of [n][k]; its tiles are
   // loaded as 64x64 boxes and consumed as an N-major MMA operand.
   // sym_ops (bit 0: P, bit 1: Q): the operand is a symmetric matrix stored only
@@ -450,10 +447,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           }
         } else {
           tma_store_3d(buf, &mapDst, j0, c.ti * kBM, c.b);
-          if (c.mirror && ep.dst_t != nullptr) {
-            tma_store_3d(buf + kSlabBytes, &mapDstT, c.ti * kBM, j0, c.b);
-            tma_store_3d(buf + kSlabBytes + kSlabBytes / 2, &mapDstT, c.ti * kBM + 64, j0, c.b);
-          }
         }
         tma_store_commit();
         if (g + kEpiBufs < n_slabs) {
@@ -494,7 +487,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
         const float f = ep.alpha_pow == 2 ? al * al : (ep.alpha_pow == 1 ? al : 1.f);
         const float ka = f * ep.k_acc, kx = f * ep.k_aux;
         const float kx2 = AUX2 ? f * ep.k_aux2 : 0.f;
-        const bool write_t = c.mirror && ep.dst_t != nullptr;
 #pragma unroll 1
         for (int sl = 0; sl < kSlabs; ++sl, ++g) {
           const int bsel = g % kEpiBufs;
@@ -569,14 +561,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
               }
             }
             *p = outv;
-            if (write_t) {
-              const __nv_bfloat16* o1 = reinterpret_cast<const __nv_bfloat16*>(&outv);
-#pragma unroll
-              for (int k = 0; k < 8; ++k) {
-                const uint32_t cc = half * 32 + v * 8 + k;     // column inside the slab = row of the transpose
-                *reinterpret_cast<__nv_bfloat16*>(tbuf + sw128(cc, rt >> 3) + (rt & 7) * 2) = o1[k];
-              }
-            }
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
@@ -598,7 +582,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
 #pragma unroll
           for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r[e]);
           aux_unpack<32>(aux[ch & 1], x);
-          epilogue_row<__nv_bfloat16, 32>(ep, c.b, i, jbase + ch * 32, v, c.mirror, x);
+          epilogue_row<__nv_bfloat16, 32>(ep, c.b, i, jbase + ch * 32, v, x);
         }
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -757,7 +741,7 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
                            cudaStream_t stream, int64_t* launches) {
   if (!tc) return cudaErrorInvalidValue;
   if (pb.Mp % kBN != 0 || pb.Np % kBN != 0 || pb.Kp % kBK != 0) return cudaErrorInvalidValue;
-  CUtensorMap mp, mq, maux, maux2, mdst, mdt, msp, msq;
+  CUtensorMap mp, mq, maux, maux2, mdst, msp, msq;
   if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
   if (!pb.q_mn) {
     if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
@@ -766,8 +750,8 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
     if (pb.symmetric || !get_map(tc, pb.Q, pb.Kp, pb.Np, pb.batch, 64, &mq)) return cudaErrorInvalidValue;
   }
   // Epilogue maps (product epilogues only): auxiliary and result slabs of 128
-  // rows x 64 columns, transposed result in boxes of 64 x 64.
-  maux = mp; maux2 = mp; mdst = mp; mdt = mp; msp = mp; msq = mp;
+  // rows x 64 columns.
+  maux = mp; maux2 = mp; mdst = mp; msp = mp; msq = mp;
   // 64x64 boxes over a symmetric operand, through which its mirrored blocks are read
   if (pb.sym_ops & 1) {
     if (pb.Mp != pb.Kp || !get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, 64, &msp)) return cudaErrorInvalidValue;
@@ -781,17 +765,13 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   }
   if (ep.aux2) {
     // second auxiliary operand: product epilogues of two symmetric operands only
-    if (ep.kind != 0 || !ep.aux || ep.dst_t || pb.q_mn || pb.sym_ops != 3) return cudaErrorInvalidValue;
+    if (ep.kind != 0 || !ep.aux || pb.q_mn || pb.sym_ops != 3) return cudaErrorInvalidValue;
     if (ep.bs_aux2 != pb.Mp * ep.ld_aux2) return cudaErrorInvalidValue;
     if (!get_map(tc, ep.aux2, pb.Mp, ep.ld_aux2, pb.batch, 128, &maux2)) return cudaErrorInvalidValue;
   }
   if (ep.kind == 0) {
     if (ep.bs_dst != pb.Mp * ep.ld_dst) return cudaErrorInvalidValue;
     if (!get_map(tc, ep.dst, pb.Mp, ep.ld_dst, pb.batch, 128, &mdst)) return cudaErrorInvalidValue;
-    if (ep.dst_t) {
-      if (ep.bs_dst_t != pb.Np * ep.ld_dst_t) return cudaErrorInvalidValue;
-      if (!get_map(tc, ep.dst_t, pb.Np, ep.ld_dst_t, pb.batch, 64, &mdt)) return cudaErrorInvalidValue;
-    }
   }
   const int64_t mt = pb.Mp / kBM, nt = pb.Np / kBN;
   int64_t per_mat;
@@ -820,7 +800,7 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   cfg.numAttrs = 1;
   const int kt = (int)(pb.Kp / kBK);
 #define PRM_TC_LAUNCH(QMN, SYM, AX2)                                                                              \
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<QMN, SYM, AX2>, mp, mq, maux, maux2, mdst, mdt, msp, msq, kt,     \
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<QMN, SYM, AX2>, mp, mq, maux, maux2, mdst, msp, msq, kt,          \
                             (int)per_mat, (int)total, pb.symmetric, (int)mt, ep, status)
   if (pb.q_mn && pb.sym_ops == 1) PRM_TC_LAUNCH(1, 1, 0);
   if (pb.q_mn && !pb.sym_ops) PRM_TC_LAUNCH(1, 0, 0);

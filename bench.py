@@ -44,7 +44,8 @@ ROW_DRAM_BYTES_PER_ELEMENT = 14.0   # wide; the captures never exceed the algori
 def ns5_flops(shapes, exec_flop=None):
     """(executed, paper model) flop of one refresh.  Executed: what the library
     reports per matrix of each shape (exec_flop: {shape: flop}, from
-    prm_group_info: 9r^2c+11r^3 where the first iterations run in Gram space), else the printed recurrence with triangle-only symmetric
+    prm_group_info: 9r^2c+11r^3 or 8r^2c+13r^3 where the first iterations run in
+    Gram space), else the printed recurrence with triangle-only symmetric
     products, 15r^2c+5r^3."""
     ex = mo = 0
     for (m, n) in shapes:
@@ -241,7 +242,7 @@ def run_sharded(args, wl, K, rank, local_rank, world, dev):
     n = len(shapes)
     dist = world > 1
     opt = B.PeriodicRowwiseMuon(shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma, io_dtype=wl.io_dtype,
-                                gram_span=not args.printed_ns5, device=dev)
+                                gram_span=0 if args.printed_ns5 else args.ns5_schedule, device=dev)
 
     def shard(t, rows):
         lo, cnt = B.prm_shard_rows(rows, world, rank)
@@ -362,7 +363,10 @@ def main():
     ap.add_argument("--check-mode", action="store_true", help="NS5 in fp32 on CUDA cores")
     ap.add_argument("--first-step", type=int, default=None, help="step index of the first warm-up step")
     ap.add_argument("--printed-ns5", action="store_true",
-                    help="all five NS5 iterations as printed (no Gram-space iterations)")
+                    help="all five NS5 iterations as printed (no Gram-space iterations); same as --ns5-schedule 0")
+    ap.add_argument("--ns5-schedule", type=int, default=2, choices=[0, 1, 2],
+                    help="PRM_OPT_NS_GRAM_SPAN: 0 printed recurrence, 1 first three iterations in Gram space, "
+                         "2 (library default) also the last Gram matrix from the one before it")
     ap.add_argument("--sharded", action="store_true",
                     help="the paper's distributed execution over the N ranks (rows sharded, bucketed all-gather "
                          "refresh, sharded tall RowNorm) instead of N independent replicas")
@@ -402,7 +406,7 @@ def main():
     n = len(wl.shapes)
     io_bytes = 4 if wl.io_dtype == "fp32" else 2
     opt = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
-                                io_dtype=wl.io_dtype, check_mode=args.check_mode, gram_span=not args.printed_ns5,
+                                io_dtype=wl.io_dtype, check_mode=args.check_mode, gram_span=0 if args.printed_ns5 else args.ns5_schedule,
                                 device=dev)
     gram_iters = {(g["rows"], g["cols"]): g["gram_iters"] for g in opt.groups()}
     exec_flop = {(g["rows"], g["cols"]): g["ns5_flop"] for g in opt.groups()}
@@ -511,8 +515,10 @@ def main():
                    "elements": el, "io_dtype": wl.io_dtype, "momentum_dtype": "fp32",
                    "ns5": "fp32 check mode" if args.check_mode else "bf16 tcgen05",
                    "ns5_schedule": ("five iterations as printed" if not any(gram_iters.values()) else
-                                    "iterations 1-3 in Gram space for %d of %d matrices, 4-5 as printed" % (
-                                        sum(1 for sh in wl.shapes if gram_iters.get(tuple(sh), 0)), n)),
+                                    "PRM_OPT_NS_GRAM_SPAN=%d: iterations 1-3 in Gram space for %d of %d matrices%s" % (
+                                        args.ns5_schedule, sum(1 for sh in wl.shapes if gram_iters.get(tuple(sh), 0)), n,
+                                        ", last Gram matrix from the previous one where c > 2r"
+                                        if args.ns5_schedule == 2 else "")),
                    "replicas": world, "l2": "inputs larger than L2 (working set %.1f GB)" % (el * 8 / 1e9),
                    "first_timed_step_index": t_first + args.warmup},
         "refresh_ms": mean_ref if n_ref else None, "row_step_ms": mean_row if n_row else None,

@@ -71,15 +71,22 @@ extern "C" {
 #define PRM_OPT_NO_REFRESH  11  /* 1: RowNorm at every step, no NS5 schedule; default 0 */
 /* How the tensor-core path evaluates the five NS5 iterations (Appendix "Cost of
  * NS5").  The iteration X <- aX + BX with A = X X^T, B = bA + cA^2 keeps every A_k
- * a polynomial in A_0, and A_{k+1} = (aI + B_k) A_k (aI + B_k).  1 (default): for
- * matrices with at least 1024 oriented rows r and c >= 1.5 r columns the first
- * three iterations work on r x r matrices only (A_1, A_2 and the product of the
- * three factors aI + B_k from r x r products), then X_3 comes from one r x c
- * product and the last two iterations run as printed: 9 r^2 c + 11 r^3 flop
- * instead of 15 r^2 c + 5 r^3, the same result in exact arithmetic.  0: all five
- * iterations as printed.  The check mode always runs them as printed.  Before
- * set_workspace (the workspace holds two more r x r matrices per refreshed
- * matrix when this is on). */
+ * a polynomial in A_0, and A_{k+1} = (aI + B_k) A_k (aI + B_k).
+ *   0: all five iterations as printed, 15 r^2 c + 5 r^3 flop per matrix (with
+ *      triangle-only symmetric products).
+ *   1: for matrices with at least 1024 oriented rows r and c >= 1.5 r columns
+ *      the first three iterations work on r x r matrices only (A_1, A_2 and the
+ *      product of the three factors aI + B_k from r x r products), then X_3
+ *      comes from one r x c product and the last two iterations run as
+ *      printed: 9 r^2 c + 11 r^3 flop, the same result in exact arithmetic and
+ *      the same measured error as 0.
+ *   2 (default): as 1, and beyond c = 2 r the Gram matrix of the fifth iteration
+ *      is taken from the fourth's (A_4 = (aI + B_3) A_3 (aI + B_3), two r x r
+ *      products instead of X_4 X_4^T): 8 r^2 c + 13 r^3 flop.  Measured error
+ *      against the fp64 recurrence 5-50 % above that of 0 and 1 on the
+ *      benchmark's inputs (at most 1.1e-2 relative Frobenius error).
+ * The check mode always runs the iterations as printed.  Before set_workspace
+ * (the workspace holds two more r x r matrices per refreshed matrix with 1 or 2). */
 #define PRM_OPT_NS_GRAM_SPAN 12
 
 

@@ -349,7 +349,7 @@ class PeriodicRowwiseMuon:
 
     def __init__(self, shapes, K, beta=0.95, nesterov=False, lr=5e-3, wd=0.01, *, gamma=0.15,
                  eps_row=1e-8, eps_ns=1e-7, scale_mode=1, io_dtype="bf16", check_mode=False,
-                 ns_workspace_bytes=None, gamma_ns=1.0, no_refresh=False, gram_span=True, device="cuda"):
+                 ns_workspace_bytes=None, gamma_ns=1.0, no_refresh=False, gram_span=2, device="cuda"):
         self.shapes = [(int(m), int(n)) for (m, n) in shapes]
         self.device = torch.device(device)
         self.io_dtype = io_dtype
@@ -364,7 +364,7 @@ class PeriodicRowwiseMuon:
             prm_set_option(self.h, PRM_OPT_CHECK_MODE, 1 if check_mode else 0)
             prm_set_option(self.h, PRM_OPT_GAMMA_NS, gamma_ns)
             prm_set_option(self.h, PRM_OPT_NO_REFRESH, 1 if no_refresh else 0)
-            prm_set_option(self.h, PRM_OPT_NS_GRAM_SPAN, 1 if gram_span else 0)
+            prm_set_option(self.h, PRM_OPT_NS_GRAM_SPAN, int(gram_span))
             if ns_workspace_bytes is not None:
                 prm_set_option(self.h, PRM_OPT_NS_WORKSPACE_BYTES, ns_workspace_bytes)
             nbytes = prm_workspace_bytes(self.h)

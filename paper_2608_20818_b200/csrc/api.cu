@@ -25,7 +25,7 @@ struct prm_ctx {
   size_t ns_cap = (size_t)8 << 30;
   float gamma_ns = 1.f;   // multiplier on the NS5 branch (ablation: "scalar-controlled" uses gamma)
   int no_refresh = 0;     // ablation: RowNorm at every step
-  int gram_span = 1;      // first NS5 iterations in Gram space where it pays (tensor-core path)
+  int gram_span = 2;      // NS5 schedule of the tensor-core path (PRM_OPT_NS_GRAM_SPAN)
 
   std::vector<Group> groups;
   std::vector<int> group_of_mat, order_in_group, slot_of_mat;   // slot = index in pointer tables
@@ -116,6 +116,9 @@ static void compute_layout(prm_ctx* c) {
     // from c = 1.5 r on; below 1024 rows the time is noise and the bf16 rounding of the
     // small r x r matrices averages less well, so those stay on the printed recurrence.
     g.gram_iters = (!c->check_mode && c->gram_span && g.rp >= 1024 && 2 * g.cp >= 3 * g.rp) ? kGramIters : 0;
+    // Mode 2: beyond c = 2r the Gram matrix of the last iteration is also cheaper from the one
+    // before it (A_4 = P_3 A_3 P_3, two r^3 products) than from X_4 (one r^2 c product).
+    g.last_gram_rec = (g.gram_iters && c->gram_span >= 2 && g.cp > 2 * g.rp) ? 1 : 0;
     // X ping-pong, A, B (+ two more r x r matrices for the Gram-space iterations)
     const size_t per_mat = e * (size_t)(2 * g.rp * g.cp + (g.gram_iters ? 4 : 2) * g.rp * g.rp);
     int nb = (int)std::min<size_t>((size_t)g.count, std::max<size_t>(1, c->ns_cap / per_mat));
@@ -209,8 +212,13 @@ extern "C" int prm_set_option(prm_ctx* c, int key, double v) {
         if (v < 0) return fail(c, PRM_ERR_ARG, "workspace cap must be >= 0");
         c->ns_cap = (size_t)v;
       } else {
-        if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
-        (key == PRM_OPT_IO_DTYPE ? c->io_fp32 : key == PRM_OPT_CHECK_MODE ? c->check_mode : c->gram_span) = (int)v;
+        if (key == PRM_OPT_NS_GRAM_SPAN) {
+          if (v != 0 && v != 1 && v != 2) return fail(c, PRM_ERR_ARG, "value must be 0, 1 or 2");
+          c->gram_span = (int)v;
+        } else {
+          if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
+          (key == PRM_OPT_IO_DTYPE ? c->io_fp32 : c->check_mode) = (int)v;
+        }
       }
       compute_layout(c);
       return PRM_OK;
@@ -260,9 +268,9 @@ extern "C" int prm_group_info(const prm_ctx* c, int group, int64_t* rows, int64_
   if (ns5_flop) {
     // X X^T products (r^2 c each, lower blocks), r x c products (2 r^2 c), symmetric r x r products (r^3)
     const double r = (double)g.r, cc = (double)g.c;
-    const double n_gram = g.gram_iters ? 3 : 5;
+    const double n_gram = g.gram_iters ? (g.last_gram_rec ? 2 : 3) : 5;
     const double n_rc = g.gram_iters ? 3 : 5;
-    const double n_rr = g.gram_iters ? 11 : 5;
+    const double n_rr = g.gram_iters ? (g.last_gram_rec ? 13 : 11) : 5;
     *ns5_flop = n_gram * r * r * cc + n_rc * 2.0 * r * r * cc + n_rr * r * r * r;
   }
   return PRM_OK;
@@ -353,14 +361,17 @@ static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFina
     it0 = kGramIters;
   }
   for (int it = it0; it < kNsIters && ce == cudaSuccess; ++it) {
-    // A = X X^T (times alpha^2 in the first iteration)
-    GemmProblem pa;
-    pa.P = X[cur]; pa.Q = X[cur]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
-    pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
-    Epilogue ea;
-    ea.dst = A; ea.ld_dst = g.rp; ea.bs_dst = rr;   // blocks on and below the diagonal only
-    if (it == 0) { ea.alpha = alpha; ea.alpha_pow = 2; }
-    if ((ce = gemm(pa, ea, PRM_PROF_GRAM)) != cudaSuccess) break;
+    // A = X X^T (times alpha^2 in the first iteration), unless the previous iteration already
+    // produced it from its own Gram matrix
+    if (!(g.last_gram_rec && it == kNsIters - 1)) {
+      GemmProblem pa;
+      pa.P = X[cur]; pa.Q = X[cur]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
+      pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
+      Epilogue ea;
+      ea.dst = A; ea.ld_dst = g.rp; ea.bs_dst = rr;   // blocks on and below the diagonal only
+      if (it == 0) { ea.alpha = alpha; ea.alpha_pow = 2; }
+      if ((ce = gemm(pa, ea, PRM_PROF_GRAM)) != cudaSuccess) break;
+    }
     // B = b A + c A^2
     GemmProblem pp;
     pp.P = A; pp.Q = A; pp.Mp = g.rp; pp.Np = g.rp; pp.Kp = g.rp;
@@ -369,6 +380,22 @@ static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFina
     eb.k_acc = kNsC; eb.k_aux = kNsB; eb.aux = A; eb.ld_aux = g.rp; eb.bs_aux = rr;
     eb.dst = B; eb.ld_dst = g.rp; eb.bs_dst = rr;
     if ((ce = gemm(pp, eb, PRM_PROF_POLY)) != cudaSuccess) break;
+    if (g.last_gram_rec && it == kNsIters - 2) {
+      // A_4 = (aI + B_3) A_3 (aI + B_3) from r x r products: Z = aA_3 + A_3 B_3, then A_4 = aZ + Z B_3.
+      // X_4 is still formed below with B_3; only the Gram matrix of the last iteration is not
+      // recomputed from the rounded X_4.
+      auto step = [&](const char* Pm, char* dst) -> cudaError_t {
+        GemmProblem pb;
+        pb.P = Pm; pb.Q = B; pb.Mp = g.rp; pb.Np = g.rp; pb.Kp = g.rp;
+        pb.bs_P = rr; pb.bs_Q = rr; pb.batch = nb; pb.symmetric = 1; pb.sym_ops = 3;
+        Epilogue ep;
+        ep.k_acc = 1.f; ep.k_aux = kNsA; ep.aux = Pm; ep.ld_aux = g.rp; ep.bs_aux = rr;
+        ep.dst = dst; ep.ld_dst = g.rp; ep.bs_dst = rr;
+        return gemm(pb, ep, PRM_PROF_GRAMSPACE);
+      };
+      if ((ce = step(A, R[2])) != cudaSuccess) break;
+      if ((ce = step(R[2], A)) != cudaSuccess) break;       // A_3 is no longer needed: A now holds A_4
+    }
     // X <- a X + B X (times alpha in the first iteration); last iteration
     // goes straight into the parameters.
     GemmProblem pu;

@@ -157,6 +157,7 @@ struct Group {
   int64_t rp = 0, cp = 0;       // padded oriented shape (NS5 workspace)
   int ns_batch = 1;             // matrices refreshed per sub-batch
   int gram_iters = 0;           // leading NS5 iterations run in Gram space (0 or kGramIters)
+  int last_gram_rec = 0;        // 1: the last iteration's Gram matrix comes from the previous one's
   size_t tall_scratch_off = 0;  // byte offset of column partials (tall groups)
   size_t tall_nu_off = 0;       // byte offset of column norms (tall groups)
 };

@@ -108,17 +108,19 @@ def test_group_info_and_gram_span_option():
     # Gram-space iterations: >= 1024 oriented rows and c >= 1.5 r (padded to 256)
     assert [g["gram_iters"] for g in info] == [3, 0, 3, 0, 0]
     d = 2048.0
-    assert [g["ns5_flop"] for g in info[:3]] == [9 * d * d * 6144 + 11 * d ** 3, 20 * d ** 3, 9 * d * d * 8192 + 11 * d ** 3]
+    assert [g["ns5_flop"] for g in info[:3]] == [8 * d * d * 6144 + 13 * d ** 3, 20 * d ** 3, 8 * d * d * 8192 + 13 * d ** 3]
     assert all(g["ns_batch"] == g["count"] for g in info)
     with_span = B.prm_workspace_bytes(h)
     B.prm_set_option(h, B.PRM_OPT_NS_GRAM_SPAN, 0)
     assert [B.prm_group_info(h, g)["gram_iters"] for g in range(n_groups)] == [0] * 5
     assert B.prm_workspace_bytes(h) < with_span
     B.prm_set_option(h, B.PRM_OPT_NS_GRAM_SPAN, 1)
+    assert B.prm_group_info(h, 0)["ns5_flop"] == 9 * d * d * 6144 + 11 * d ** 3
+    assert B.prm_workspace_bytes(h) == with_span
     B.prm_set_option(h, B.PRM_OPT_CHECK_MODE, 1)          # the check mode runs the printed recurrence
     assert [B.prm_group_info(h, g)["gram_iters"] for g in range(n_groups)] == [0] * 5
     with pytest.raises(B.PrmError) as e:
-        B.prm_set_option(h, B.PRM_OPT_NS_GRAM_SPAN, 2)
+        B.prm_set_option(h, B.PRM_OPT_NS_GRAM_SPAN, 3)
     assert e.value.code == B.PRM_ERR_ARG
     with pytest.raises(B.PrmError) as e:
         B.prm_group_info(h, n_groups)

@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 SHAPES = [(256, 1024), (24, 40), (40, 24), (300, 520), (512, 256), (5, 5), (1, 9), (130, 1000), (768, 768)]
 
 
-def _direction_case(shapes, io, check_mode, seed, nesterov=True, ns_ws=None, gram_span=True):
+def _direction_case(shapes, io, check_mode, seed, nesterov=True, ns_ws=None, gram_span=2):
     """W = 0, lr = 1, wd = 0: the step writes -s * NS5 direction."""
     cfg = U.oracle_cfg(K=3, beta=0.95, nesterov=nesterov, lr=1.0, wd=0.0, scale_mode=0)
     W, G, M = U.make_inputs(shapes, seed, io, grad_std=1e-3, mom_std=1e-3)

@@ -25,63 +25,71 @@ CASES = [((1024, 3072), 3), ((4096, 1024), 3), ((1024, 2048), 3), ((2048, 1024),
 
 @pytest.mark.parametrize("shape,iters", CASES)
 def test_gramspace_direction_within_bound_and_eligibility(shape, iters):
-    opt = B.PeriodicRowwiseMuon([shape], 1)
-    assert opt.groups()[0]["gram_iters"] == iters
-    opt.close()
-    opt = B.PeriodicRowwiseMuon([shape], 1, gram_span=False)
-    assert opt.groups()[0]["gram_iters"] == 0
-    opt.close()
-    (err,) = _direction_case([shape], "bf16", False, seed=sum(shape))
-    (err_printed,) = _direction_case([shape], "bf16", False, seed=sum(shape), gram_span=False)
-    assert err <= TOL and err_printed <= TOL, (err, err_printed)
+    for mode, want in ((2, iters), (1, iters), (0, 0)):
+        opt = B.PeriodicRowwiseMuon([shape], 1, gram_span=mode)
+        assert opt.groups()[0]["gram_iters"] == want
+        opt.close()
+    errs = [_direction_case([shape], "bf16", False, seed=sum(shape), gram_span=mode)[0] for mode in (0, 1, 2)]
+    assert max(errs) <= TOL, errs
+    r, c = min(shape), max(shape)
+    r_p, c_p = -(-r // 256) * 256, -(-c // 256) * 256
     if iters == 0:
-        assert err == err_printed
+        assert errs[0] == errs[1] == errs[2]
+    elif c_p <= 2 * r_p:
+        assert errs[1] == errs[2]          # the last Gram matrix is recomputed unless c > 2r
 
 
 def test_gramspace_launch_classes_and_sub_batches():
+    # (1024, 2560): c > 2r, so mode 2 takes the last Gram matrix from the one before it
     shapes = [(1024, 2048)] * 3 + [(2048, 1024)] * 2 + [(512, 1024)] + [(1024, 2560)]
     cfg = U.oracle_cfg(K=1, nesterov=True, lr=1.0, wd=0.0, scale_mode=0)
     W, G, M = U.make_inputs(shapes, 17, "bf16", grad_std=1e-3, mom_std=1e-3)
     for w in W:
         w.zero_()
-    for ns_ws, sub_batches in ((None, (1, 1, 1, 1)), (1, (3, 2, 1, 1))):
-        opt = B.PeriodicRowwiseMuon(shapes, 1, 0.95, True, 1.0, 0.0, scale_mode=0, ns_workspace_bytes=ns_ws)
-        info = opt.groups()
-        assert [g["gram_iters"] for g in info] == [3, 3, 0, 3]
-        r, c = 1024.0, 2560.0
-        assert info[3]["ns5_flop"] == 9 * r * r * c + 11 * r ** 3
-        assert info[0]["ns5_flop"] == 9 * r * r * 2048 + 11 * r ** 3
-        assert info[2]["ns5_flop"] == 15 * 512.0 ** 2 * 1024 + 5 * 512.0 ** 3
-        w = [x.cuda() for x in W]
-        g = [x.cuda() for x in G]
-        m = [x.cuda() for x in M]
-        opt.profile(True)
-        opt.step(w, g, m, 0)
-        prof = opt.profile_read()
-        torch.cuda.synchronize()
-        assert opt.status() == B.PRM_OK
-        n_gram = sub_batches[0] + sub_batches[1]          # sub-batches refreshed in Gram space
-        n_printed = sub_batches[2]
-        n_gram += sub_batches[3]
-        assert prof["gramspace"][1] == 6 * n_gram
-        assert prof["gram"][1] == 3 * n_gram + 5 * n_printed
-        assert prof["poly"][1] == 5 * (n_gram + n_printed)
-        assert prof["update"][1] == 2 * n_gram + 4 * n_printed
-        assert prof["update_final"][1] == n_gram + n_printed
-        for i, s in enumerate(shapes):
-            Wr, _ = O.step_matrix(U.to_np64(W[i]), U.to_np64(G[i]), U.to_np64(M[i]), 0, cfg)
-            assert U.rel_fro(U.to_np64(w[i]), Wr) <= TOL, (i, s)
-        opt.close()
+    for mode in (1, 2):
+        for ns_ws, sub_batches in ((None, (1, 1, 1, 1)), (1, (3, 2, 1, 1))):
+            opt = B.PeriodicRowwiseMuon(shapes, 1, 0.95, True, 1.0, 0.0, scale_mode=0, ns_workspace_bytes=ns_ws,
+                                        gram_span=mode)
+            info = opt.groups()
+            assert [g["gram_iters"] for g in info] == [3, 3, 0, 3]
+            r, c = 1024.0, 2560.0
+            assert info[3]["ns5_flop"] == (8 * r * r * c + 13 * r ** 3 if mode == 2 else 9 * r * r * c + 11 * r ** 3)
+            assert info[0]["ns5_flop"] == 9 * r * r * 2048 + 11 * r ** 3
+            assert info[2]["ns5_flop"] == 15 * 512.0 ** 2 * 1024 + 5 * 512.0 ** 3
+            w = [x.cuda() for x in W]
+            g = [x.cuda() for x in G]
+            m = [x.cuda() for x in M]
+            opt.profile(True)
+            opt.step(w, g, m, 0)
+            prof = opt.profile_read()
+            torch.cuda.synchronize()
+            assert opt.status() == B.PRM_OK
+            n_gram = sub_batches[0] + sub_batches[1]          # sub-batches refreshed in Gram space
+            n_printed = sub_batches[2]
+            n_rec = 0
+            if mode == 2:
+                n_rec = sub_batches[3]                        # ... and with the last Gram matrix by recurrence
+            else:
+                n_gram += sub_batches[3]
+            assert prof["gramspace"][1] == 6 * n_gram + 8 * n_rec
+            assert prof["gram"][1] == 3 * n_gram + 5 * n_printed + 2 * n_rec
+            assert prof["poly"][1] == 5 * (n_gram + n_printed + n_rec)
+            assert prof["update"][1] == 2 * (n_gram + n_rec) + 4 * n_printed
+            assert prof["update_final"][1] == n_gram + n_printed + n_rec
+            for i, s in enumerate(shapes):
+                Wr, _ = O.step_matrix(U.to_np64(W[i]), U.to_np64(G[i]), U.to_np64(M[i]), 0, cfg)
+                assert U.rel_fro(U.to_np64(w[i]), Wr) <= TOL, (i, s)
+            opt.close()
 
 
 @pytest.mark.parametrize("kind", ["heavy_rows", "low_rank_mild"])
 def test_gramspace_structured_inputs(kind):
-    errs = _structured_case(kind, [(1024, 2048), (2048, 1024)], False)
+    errs = _structured_case(kind, [(1024, 2048), (2048, 1024), (1024, 3072), (3072, 1024)], False)
     assert max(errs) <= TOL, errs
 
 
 def test_gramspace_spiked_spectrum_no_worse_than_printed_bound():
-    errs = _structured_case("spiked", [(1024, 2048)], False)
+    errs = _structured_case("spiked", [(1024, 2048), (1024, 3072)], False)
     assert max(errs) <= 0.1, errs
 
 

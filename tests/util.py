@@ -53,7 +53,7 @@ def oracle_cfg(**kw):
 
 
 def gpu_step(shapes, W, G, M, t, cfg, io, check_mode, ns_workspace_bytes=None, steps=1, grads_fn=None,
-             gram_span=True):
+             gram_span=2):
     """Run `steps` steps from step index t on the GPU through the C ABI.
     Returns (W_new list, M_new list) as fp64 numpy, after checking canaries."""
     opt = B.PeriodicRowwiseMuon(shapes, cfg.K, cfg.beta, cfg.nesterov, cfg.lr, cfg.wd, gamma=cfg.gamma,

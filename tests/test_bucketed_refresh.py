@@ -442,3 +442,31 @@ def test_partition_matrices_is_balanced_and_deterministic():
     assert B.prm_partition_matrices([(4, 4)], 3)[0] == [0]
     with pytest.raises(B.PrmError):
         B.prm_partition_matrices([(4, 4)], 0)
+
+
+def test_planning_functions_on_random_inputs():
+    from hypothesis import given, settings, strategies as st
+
+    shape = st.tuples(st.integers(1, 5000), st.integers(1, 5000))
+
+    @settings(max_examples=150, deadline=None)
+    @given(st.lists(shape, min_size=1, max_size=12), st.integers(1, 9), st.integers(1, 1 << 26))
+    def plan(shapes, world, cap):
+        want = O.bucket_plan(shapes, world, cap)
+        got = B.prm_bucket_plan(shapes, world, cap)
+        assert list(got[0]) == want[0] and list(got[1]) == want[1] and list(got[2]) == want[2]
+        _check_plan(shapes, world, cap, got)
+
+    @settings(max_examples=150, deadline=None)
+    @given(st.integers(1, 1 << 20), st.integers(1, 64))
+    def rows(n, world):
+        covered = 0
+        for q in range(world):
+            lo, cnt = B.prm_shard_rows(n, world, q)
+            assert (lo, cnt) == O.shard_rows(n, world, q)
+            assert lo == min(n, covered) and cnt >= 0
+            covered += cnt
+        assert covered == n
+
+    plan()
+    rows()

@@ -695,6 +695,8 @@ TcContext* tc_create(std::string* err) {
 void tc_destroy(TcContext* tc) { delete tc; }
 
 // 3-D map over a [batch][rows][kdim] bf16 array; box = 64 (k) x box_rows x 1.
+// No L2 promotion: every 128-byte row of a box is used whole, and the refresh of
+// the 9B-class set measured 0.5-0.7 % faster without the 256-byte promotion.
 static bool get_map(TcContext* tc, const void* base, int64_t rows, int64_t kdim, int batch, int box_rows,
                     CUtensorMap* out) {
   auto key = std::make_tuple(base, rows, kdim, batch, box_rows);
@@ -706,7 +708,7 @@ static bool get_map(TcContext* tc, const void* base, int64_t rows, int64_t kdim,
   cuuint32_t estr[3] = {1, 1, 1};
   CUresult r = tc->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
                           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return false;
   if (tc->cache.size() > 4096) tc->cache.clear();
   tc->cache[key] = *out;

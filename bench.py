@@ -270,7 +270,8 @@ def run_sharded(args, wl, K, rank, local_rank, world, dev):
 
     def step(t):
         if t % K == 0:
-            S.bucketed_refresh_step(shapes, params, grads, moms, refresh_backend, bucket_bytes=cap, buffers=buffers)
+            S.bucketed_refresh_step(shapes, params, grads, moms, refresh_backend, bucket_bytes=cap, buffers=buffers,
+                                    exchange=args.exchange)
         else:
             S.sharded_row_step(tall, wide_step, tall_backend, stream=stream.cuda_stream)
 
@@ -306,6 +307,9 @@ def run_sharded(args, wl, K, rank, local_rank, world, dev):
     # per-bucket times in isolation: gather alone, then rebuild + NS5 + slice alone
     bucket_of_mat, offsets, segments = B.prm_bucket_plan(shapes, world, cap)
     a_ms, c_ms = [], []
+    if args.exchange == "p2p":          # no separate transfer to time: the rebuild does the reading
+        buffers = {"send": buffers["send"],
+                   "recv": [torch.empty(max(segments) * world, dtype=torch.bfloat16, device=dev)]}
     for l, seg in enumerate(segments):
         members = [i for i in range(n) if bucket_of_mat[i] == l]
         send = buffers["send"][0][:seg]
@@ -338,7 +342,7 @@ def run_sharded(args, wl, K, rank, local_rank, world, dev):
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": wl.name, "K": K, "matrices": n, "blocks": wl.blocks, "d": wl.d,
                    "parallelism": "rows sharded over %d ranks (Algorithm 2), NS5 replicated" % world,
-                   "bucket_mib": args.bucket_mib, "buckets": len(segments),
+                   "bucket_mib": args.bucket_mib, "buckets": len(segments), "exchange": args.exchange,
                    "l2": "inputs larger than L2"},
         "refresh_ms": mean_ref if ref_ms else None, "row_step_ms": mean_row if row_ms else None,
         "clocks": clocks,
@@ -371,6 +375,9 @@ def main():
                     help="the paper's distributed execution over the N ranks (rows sharded, bucketed all-gather "
                          "refresh, sharded tall RowNorm) instead of N independent replicas")
     ap.add_argument("--bucket-mib", type=int, default=240, help="--sharded: cap on one bucket's gathered payload")
+    ap.add_argument("--exchange", default="allgather", choices=["allgather", "p2p"],
+                    help="--sharded: NCCL all-gather per bucket, or no collective: the rebuild reads every rank's "
+                         "segment in place through symmetric memory (peer loads over NVLink)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -342,6 +342,16 @@ PRM_API int prm_tall_shard_apply(void* param_shard, const void* grad_shard, cons
  *   after the call's work completes.  mats, offsets and param_shards are HOST
  *   arrays.  Errors as for prm_step; PRM_ERR_SHAPE if a matrix does not fit
  *   its segment.
+ * prm_refresh_segments      the same, but the world segments are given by
+ *   their own device pointers (HOST array of world pointers, 2-byte aligned,
+ *   16-byte aligned for vector loads; at most 64 ranks).  A pointer may map
+ *   ANOTHER GPU's memory (CUDA IPC, symmetric memory): the rebuild then reads
+ *   the rows with plain loads over NVLink straight from the buffers the
+ *   owners packed them into, and the all-gather and its receive buffer
+ *   disappear into the pre-pass (no TMA and no multicast are involved in these
+ *   loads).  The caller orders the reads after every owner's pack (a
+ *   cross-rank barrier on the streams) and keeps a segment unchanged until all
+ *   ranks have passed the call's rebuild.
  * prm_pipeline_model  host.  Ideal two-stage pipeline over n_buckets buckets
  *   with all-gather times a[l] and compute times c[l] (Eq. app-pipeline-time,
  *   Eq. app-exposed-communication):
@@ -356,6 +366,9 @@ PRM_API int prm_shard_momentum_pack(const void* grad_shard, float* momentum_shar
                                     int64_t cols, int64_t reserved_elems, int io_fp32, float beta,
                                     int nesterov, void* u_out, void* cuda_stream);
 PRM_API int prm_refresh_gathered(prm_ctx* ctx, const int* mats, int n, const void* gathered,
+                                 int64_t segment_elems, const int64_t* offsets, int world, int rank,
+                                 void* const* param_shards, void* cuda_stream);
+PRM_API int prm_refresh_segments(prm_ctx* ctx, const int* mats, int n, const void* const* segments,
                                  int64_t segment_elems, const int64_t* offsets, int world, int rank,
                                  void* const* param_shards, void* cuda_stream);
 PRM_API int prm_pipeline_model(const double* a, const double* c, int n_buckets, double* t_pipe,

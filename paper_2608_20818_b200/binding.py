@@ -44,7 +44,7 @@ EXPORTS = (
     "prm_step_h2d", "prm_plan", "prm_status", "prm_last_error", "prm_launch_count", "prm_destroy",
     "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc", "prm_selftest_timeout", "prm_adamw_step",
     "prm_tall_shard_scratch_bytes", "prm_tall_shard_stats", "prm_tall_shard_apply", "prm_group_info",
-    "prm_shard_rows", "prm_bucket_plan", "prm_shard_momentum_pack", "prm_refresh_gathered", "prm_pipeline_model",
+    "prm_shard_rows", "prm_bucket_plan", "prm_shard_momentum_pack", "prm_refresh_gathered", "prm_refresh_segments", "prm_pipeline_model",
     "prm_partition_matrices",
 )
 PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
@@ -129,6 +129,9 @@ def lib():
     L.prm_refresh_gathered.argtypes = [c_void_p, POINTER(c_int), c_int, c_void_p, c_int64, POINTER(c_int64), c_int,
                                        c_int, POINTER(c_void_p), c_void_p]
     L.prm_refresh_gathered.restype = c_int
+    L.prm_refresh_segments.argtypes = [c_void_p, POINTER(c_int), c_int, POINTER(c_void_p), c_int64, POINTER(c_int64),
+                                       c_int, c_int, POINTER(c_void_p), c_void_p]
+    L.prm_refresh_segments.restype = c_int
     L.prm_pipeline_model.argtypes = [POINTER(c_double), POINTER(c_double), c_int, POINTER(c_double), POINTER(c_double)]
     L.prm_pipeline_model.restype = c_int
     L.prm_partition_matrices.argtypes = [POINTER(c_int64), c_int, c_int, POINTER(c_int), POINTER(c_double)]
@@ -308,6 +311,17 @@ def prm_refresh_gathered(h, mats, gathered_ptr, segment_elems, offsets, world, r
     p = (c_void_p * max(1, n))(*[c_void_p(int(x)) if x else None for x in param_shard_ptrs])
     _check(lib().prm_refresh_gathered(h, m, n, c_void_p(int(gathered_ptr)), int(segment_elems), o, int(world),
                                       int(rank), p, c_void_p(stream)), h)
+
+
+def prm_refresh_segments(h, mats, segment_ptrs, segment_elems, offsets, world, rank, param_shard_ptrs, stream):
+    """segment_ptrs: one device pointer per rank (local or peer-mapped memory)."""
+    n = len(mats)
+    m = (c_int * max(1, n))(*[int(x) for x in mats])
+    o = (c_int64 * max(1, n))(*[int(x) for x in offsets])
+    p = (c_void_p * max(1, n))(*[c_void_p(int(x)) if x else None for x in param_shard_ptrs])
+    sp = (c_void_p * max(1, int(world)))(*[c_void_p(int(x)) for x in segment_ptrs])
+    _check(lib().prm_refresh_segments(h, m, n, sp, int(segment_elems), o, int(world), int(rank), p,
+                                      c_void_p(stream)), h)
 
 
 def prm_pipeline_model(a, c):

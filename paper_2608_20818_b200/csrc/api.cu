@@ -444,18 +444,26 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
   return PRM_OK;
 }
 
-// Refresh of a bucket of matrices whose rows arrived by all-gather
+// Refresh of a bucket of matrices whose rows sit in one segment per rank
 // (Algorithm 2 lines 4-6 for one bucket, on one rank).
-extern "C" int prm_refresh_gathered(prm_ctx* c, const int* mats, int n, const void* gathered,
+extern "C" int prm_refresh_segments(prm_ctx* c, const int* mats, int n, const void* const* segments,
                                     int64_t segment_elems, const int64_t* offsets, int world, int rank,
                                     void* const* param_shards, void* cuda_stream) {
   if (!c) return PRM_ERR_ARG;
   if (!c->ws) return fail(c, PRM_ERR_WORKSPACE, "prm_refresh_gathered: no workspace attached");
-  if (n < 0 || (n > 0 && (!mats || !offsets || !param_shards || !gathered)))
+  if (n < 0 || (n > 0 && (!mats || !offsets || !param_shards || !segments)))
     return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: NULL argument");
   if (world < 1 || rank < 0 || rank >= world) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: bad world or rank");
+  if (world > kMaxWorld) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: more than 64 ranks");
   if (segment_elems < 0) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: negative segment size");
-  if (((uintptr_t)gathered & 15) != 0) return fail(c, PRM_ERR_ALIGN, "prm_refresh_gathered: buffer not 16-byte aligned");
+  SegmentPtrs segs = {};
+  bool vec_ok = true;
+  for (int q = 0; q < world && n > 0; ++q) {
+    if (!segments[q]) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: NULL segment pointer");
+    if (((uintptr_t)segments[q] & 1) != 0) return fail(c, PRM_ERR_ALIGN, "prm_refresh_gathered: segment not 2-byte aligned");
+    vec_ok = vec_ok && ((uintptr_t)segments[q] & 15) == 0;
+    segs.seg[q] = segments[q];
+  }
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   for (int k = 0; k < n; ++k) {
     if (mats[k] < 0 || mats[k] >= c->n_mats) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: matrix index out of range");
@@ -493,7 +501,7 @@ extern "C" int prm_refresh_gathered(prm_ctx* c, const int* mats, int n, const vo
       cudaError_t ce;
       {
         ProfScope ps(c, PRM_PROF_PREPASS, stream);
-        ce = launch_ns_gather_prepass(gathered, segment_elems, shard_chunk(g.rows, world), offs.data() + done, g, nb,
+        ce = launch_ns_gather_prepass(segs, vec_ok, shard_chunk(g.rows, world), offs.data() + done, g, nb,
                                       c->eps_ns, c->check_mode, c->ws + c->off_ns, fro, alpha, stream, &c->launches);
       }
       if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("gathered pre-pass: ") + cudaGetErrorString(ce));
@@ -510,6 +518,21 @@ extern "C" int prm_refresh_gathered(prm_ctx* c, const int* mats, int n, const vo
     }
   }
   return PRM_OK;
+}
+
+// The same with the segments laid out one after the other in one buffer, as an
+// all-gather delivers them.
+extern "C" int prm_refresh_gathered(prm_ctx* c, const int* mats, int n, const void* gathered,
+                                    int64_t segment_elems, const int64_t* offsets, int world, int rank,
+                                    void* const* param_shards, void* cuda_stream) {
+  if (!c) return PRM_ERR_ARG;
+  if (world < 1 || world > kMaxWorld) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: bad world (1..64)");
+  if (n > 0 && !gathered) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: NULL argument");
+  if (segment_elems < 0) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: negative segment size");
+  if (((uintptr_t)gathered & 15) != 0) return fail(c, PRM_ERR_ALIGN, "prm_refresh_gathered: buffer not 16-byte aligned");
+  const void* segs[kMaxWorld];
+  for (int q = 0; q < world; ++q) segs[q] = (const char*)gathered + (size_t)q * (size_t)segment_elems * 2;
+  return prm_refresh_segments(c, mats, n, segs, segment_elems, offsets, world, rank, param_shards, cuda_stream);
 }
 
 static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,

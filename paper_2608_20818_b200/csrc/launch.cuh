@@ -77,12 +77,15 @@ void launch_ns_alpha(const float* fro_partial, int nparts, float eps_ns, float* 
 // Refresh over row shards (Algorithm 2 lines 1-7).  Matrices of one launch
 // are described by value, kGatherMax at a time.
 constexpr int kGatherMax = 32;
+constexpr int kMaxWorld = 64;
 struct GatherBatch { int64_t off[kGatherMax]; };   // element offset of the matrix inside every rank's segment
 struct SliceBatch { void* param[kGatherMax]; };    // this rank's parameter rows
+struct SegmentPtrs { const void* seg[kMaxWorld]; }; // start of every rank's segment (local or peer memory)
 // The pre-pass on gathered rows: bf16 U of `batch` matrices of group g, read
-// from `world` segments of segment_elems elements (rank q at q*segment_elems),
-// row i of a matrix at segment i / chunk_rows, local row i % chunk_rows.
-cudaError_t launch_ns_gather_prepass(const void* gathered, int64_t segment_elems, int64_t chunk_rows,
+// from `world` segments (rank q's at segs.seg[q]): row i of a matrix comes
+// from segment i / chunk_rows, local row i % chunk_rows.  vec_ok: every
+// segment start is 16-byte aligned.
+cudaError_t launch_ns_gather_prepass(const SegmentPtrs& segs, bool vec_ok, int64_t chunk_rows,
                                      const int64_t* offs, const Group& g, int batch, float eps_ns, int x_fp32,
                                      void* X, float* fro_partial, float* alpha, cudaStream_t stream,
                                      int64_t* launches);

@@ -5,9 +5,12 @@
 //                             (Algorithm 1 line 2) and the direction input U
 //                             written as bf16 into its segment of the bucket's
 //                             send buffer
-//   (all-gather by the caller: every rank then holds all segments, rank-major)
+//   (all-gather by the caller: every rank then holds all segments, rank-major;
+//    or no copy at all: the segments stay where they were written and are
+//    read through peer-mapped pointers)
 //   ns_gather_prepass_kernel  "reconstruct full momenta": reads the rows of a
-//                             matrix from the segments they arrived in and
+//                             matrix from the segments they arrived in (or
+//                             straight from the owning GPUs' memory) and
 //                             writes the oriented, zero-padded NS5 input X with
 //                             its Frobenius partial sums; the reconstruction is
 //                             index arithmetic, no full matrix is assembled
@@ -78,15 +81,14 @@ shard_pack_scalar_kernel(const IO* __restrict__ g, float* __restrict__ m, int64_
 
 template <typename XT_, bool VEC>
 __global__ void __launch_bounds__(kThreads)
-ns_gather_prepass_kernel(const __nv_bfloat16* __restrict__ gathered, int64_t segment_elems, int chunk_rows,
-                         GatherBatch src, int rows, int cols,
+ns_gather_prepass_kernel(SegmentPtrs segs, int chunk_rows, GatherBatch src, int rows, int cols,
                          XT_* __restrict__ straight, int64_t ld_s, int64_t bs_s,
                          XT_* __restrict__ transposed, int64_t ld_t, int64_t bs_t,
                          float* __restrict__ fro_partial) {
   __shared__ float tile[kTile][kTile + 1];
   __shared__ float warp_part[kThreads / 32];
   const int b = blockIdx.z;
-  const __nv_bfloat16* __restrict__ base = gathered + src.off[b];
+  const int64_t off_b = src.off[b];
   XT_* __restrict__ ds = straight ? straight + (int64_t)b * bs_s : nullptr;
   XT_* __restrict__ dt = transposed ? transposed + (int64_t)b * bs_t : nullptr;
   const int r0 = blockIdx.y * kTile, c0 = blockIdx.x * kTile;
@@ -101,7 +103,9 @@ ns_gather_prepass_kernel(const __nv_bfloat16* __restrict__ gathered, int64_t seg
     for (int e = 0; e < 8; ++e) u[e] = 0.f;
     if (row < rows) {
       const int q = row / chunk_rows;                       // rank that sent this row
-      const __nv_bfloat16* p = base + (int64_t)q * segment_elems + (int64_t)(row - q * chunk_rows) * cols + col;
+      // plain loads: the segment may live in this GPU's memory or in a peer's
+      const __nv_bfloat16* p = reinterpret_cast<const __nv_bfloat16*>(segs.seg[q]) + off_b +
+                               (int64_t)(row - q * chunk_rows) * cols + col;
       if (VEC) {
         if (col < cols) load8_stream(p, u);
       } else {
@@ -205,14 +209,14 @@ ns_slice_update_kernel(SliceBatch dst, const XT_* __restrict__ x5, int64_t ld_x,
 }
 
 template <typename XT_>
-cudaError_t gather_prepass_inst(const __nv_bfloat16* gathered, int64_t segment_elems, int64_t chunk_rows,
+cudaError_t gather_prepass_inst(const SegmentPtrs& segs, bool vec_ok, int64_t chunk_rows,
                                 const int64_t* offs, const Group& g, int batch, float eps_ns, XT_* X,
                                 float* fro_partial, float* alpha, cudaStream_t stream, int64_t* launches) {
   const int64_t prow = g.tall ? g.cp : g.rp, pcol = g.tall ? g.rp : g.cp;
   const int64_t bs = g.rp * g.cp;
   const unsigned gx = (unsigned)(pcol / kTile), gy = (unsigned)(prow / kTile);
   if (gy > 65535) return cudaErrorInvalidValue;
-  const bool vec = (g.cols % 8 == 0) && (segment_elems % 8 == 0);
+  const bool vec = (g.cols % 8 == 0) && vec_ok;
   for (int done = 0; done < batch; done += kGatherMax) {
     const int nb = std::min(kGatherMax, batch - done);
     GatherBatch src;
@@ -227,12 +231,10 @@ cudaError_t gather_prepass_inst(const __nv_bfloat16* gathered, int64_t segment_e
     dim3 grid(gx, gy, (unsigned)nb);
     if (vec)
       ns_gather_prepass_kernel<XT_, true><<<grid, kThreads, 0, stream>>>(
-          gathered, segment_elems, (int)chunk_rows, src, (int)g.rows, (int)g.cols, straight, pcol, bs, transposed,
-          prow, bs, fp);
+          segs, (int)chunk_rows, src, (int)g.rows, (int)g.cols, straight, pcol, bs, transposed, prow, bs, fp);
     else
       ns_gather_prepass_kernel<XT_, false><<<grid, kThreads, 0, stream>>>(
-          gathered, segment_elems, (int)chunk_rows, src, (int)g.rows, (int)g.cols, straight, pcol, bs, transposed,
-          prow, bs, fp);
+          segs, (int)chunk_rows, src, (int)g.rows, (int)g.cols, straight, pcol, bs, transposed, prow, bs, fp);
     *launches += 1;
   }
   launch_ns_alpha(fro_partial, (int)(gx * gy), eps_ns, alpha, batch, stream);
@@ -269,16 +271,15 @@ cudaError_t slice_update_inst(const XT_* X5, const Group& g, int batch, void* co
 
 }  // namespace
 
-cudaError_t launch_ns_gather_prepass(const void* gathered, int64_t segment_elems, int64_t chunk_rows,
+cudaError_t launch_ns_gather_prepass(const SegmentPtrs& segs, bool vec_ok, int64_t chunk_rows,
                                      const int64_t* offs, const Group& g, int batch, float eps_ns, int x_fp32,
                                      void* X, float* fro_partial, float* alpha, cudaStream_t stream,
                                      int64_t* launches) {
-  const __nv_bfloat16* src = (const __nv_bfloat16*)gathered;
   if (x_fp32)
-    return gather_prepass_inst<float>(src, segment_elems, chunk_rows, offs, g, batch, eps_ns, (float*)X,
-                                      fro_partial, alpha, stream, launches);
-  return gather_prepass_inst<__nv_bfloat16>(src, segment_elems, chunk_rows, offs, g, batch, eps_ns,
-                                            (__nv_bfloat16*)X, fro_partial, alpha, stream, launches);
+    return gather_prepass_inst<float>(segs, vec_ok, chunk_rows, offs, g, batch, eps_ns, (float*)X, fro_partial, alpha,
+                                      stream, launches);
+  return gather_prepass_inst<__nv_bfloat16>(segs, vec_ok, chunk_rows, offs, g, batch, eps_ns, (__nv_bfloat16*)X,
+                                            fro_partial, alpha, stream, launches);
 }
 
 cudaError_t launch_ns_slice_update(const void* X5, int x_fp32, const Group& g, int batch,

@@ -134,6 +134,32 @@ class CudaRefreshBackend:
             B.prm_refresh_gathered(self.opt.h, mats, gathered.data_ptr(), segment_elems, offsets, world, rank, ptrs,
                                    stream)
 
+    def refresh_segments(self, mats, segment_ptrs, segment_elems, offsets, world, rank, param_shards, stream):
+        ptrs = [p.data_ptr() if p.numel() else 0 for p in param_shards]
+        with torch.cuda.device(self.opt.device):
+            B.prm_refresh_segments(self.opt.h, mats, segment_ptrs, segment_elems, offsets, world, rank, ptrs, stream)
+
+
+class SymmetricSendBuffers:
+    """Two send buffers of n_elems bf16 elements that every rank of the group
+    can read: torch symmetric memory (peer-mapped device memory over NVLink).
+    `ptrs(k)` are the addresses, in this process, of all ranks' k-th buffer;
+    `barrier(k)` is a cross-rank barrier enqueued on the current stream."""
+
+    def __init__(self, n_elems, device, group=None):
+        import torch.distributed as td
+        import torch.distributed._symmetric_memory as symm
+        group = group if group is not None else td.group.WORLD
+        self.n_elems = n_elems
+        self.tensors = [symm.empty(n_elems, dtype=torch.bfloat16, device=device) for _ in range(2)]
+        self.handles = [symm.rendezvous(t, group) for t in self.tensors]
+
+    def ptrs(self, k):
+        return [int(p) for p in self.handles[k].buffer_ptrs]
+
+    def barrier(self, k):
+        self.handles[k].barrier()
+
 
 def _all_gather(recv, send, group):
     import torch.distributed as td
@@ -144,7 +170,7 @@ def _all_gather(recv, send, group):
 
 
 def bucketed_refresh_step(shapes, param_shards, grad_shards, mom_shards, backend, bucket_bytes=240 << 20,
-                          group=None, world=None, rank=None, buffers=None, trace=None):
+                          group=None, world=None, rank=None, buffers=None, trace=None, exchange="allgather"):
     """One refresh step over this rank's row shards (Algorithm 2 lines 1-7).
 
     shapes        GLOBAL (rows, cols) of the Muon matrices, in the handle's order
@@ -157,9 +183,17 @@ def bucketed_refresh_step(shapes, param_shards, grad_shards, mom_shards, backend
                   buffers between calls
     trace         optional list that receives ("gather", l) / ("refresh", l)
                   in issue order
-    Work is issued on torch's current stream; the all-gather of bucket l+1 is
-    in flight while bucket l is refreshed.  Without an initialised process
-    group (or with world == 1) the exchange is a local copy.
+    exchange      "allgather": torch.distributed.all_gather_into_tensor per
+                  bucket into a receive buffer.  "p2p": no collective and no
+                  receive buffer; every rank packs into a symmetric-memory
+                  send buffer, a stream barrier follows, and the rebuild
+                  reads all ranks' segments in place with peer loads
+                  (prm_refresh_segments).  Two send buffers alternate, so one
+                  barrier per bucket orders both the reads after the packs
+                  and the next overwrite after the reads.
+    Work is issued on torch's current stream; with "allgather" the gather of
+    bucket l+1 is in flight while bucket l is refreshed.  Without an
+    initialised process group (or with world == 1) the exchange is local.
     """
     import torch.distributed as td
 
@@ -184,6 +218,11 @@ def bucketed_refresh_step(shapes, param_shards, grad_shards, mom_shards, backend
         buffers["send"] = [torch.empty(seg_max, dtype=backend.payload_dtype, device=dev) for _ in range(2)]
         buffers["recv"] = [torch.empty(seg_max * world, dtype=backend.payload_dtype, device=dev) for _ in range(2)]
     stream = torch.cuda.current_stream(dev).cuda_stream if dev.type == "cuda" else 0
+    if exchange == "p2p":
+        return _refresh_p2p(shapes, param_shards, grad_shards, mom_shards, backend, group, world, rank, buffers,
+                            trace, dist_on, (bucket_of_mat, offsets, segments), members, stream)
+    if exchange != "allgather":
+        raise ValueError("exchange must be 'allgather' or 'p2p'")
     pending = [None, None]
 
     def launch(l):                                   # lines 2 and 4: pack, then gather asynchronously
@@ -216,3 +255,41 @@ def bucketed_refresh_step(shapes, param_shards, grad_shards, mom_shards, backend
                         [param_shards[i] for i in members[l]], stream)      # line 5
         # line 6: the buffers of bucket l are reused by bucket l + 2
     return bucket_of_mat, offsets, segments
+
+
+def _refresh_p2p(shapes, param_shards, grad_shards, mom_shards, backend, group, world, rank, buffers, trace,
+                 dist_on, plan, members, stream):
+    """Algorithm 2 lines 1-7 with the all-gather folded into the rebuild: the
+    segments stay in the send buffers of their owners."""
+    bucket_of_mat, offsets, segments = plan
+    dev = param_shards[0].device
+    seg_max = max(segments)
+    key = ("p2p", seg_max, world, str(dev))
+    if buffers.get("key") != key:
+        buffers["key"] = key
+        if dist_on:
+            buffers["symm"] = SymmetricSendBuffers(seg_max, dev, group)
+            buffers["send"] = buffers["symm"].tensors
+        else:
+            buffers["symm"] = None
+            buffers["send"] = [torch.empty(seg_max, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+    symm = buffers["symm"]
+    for l, seg in enumerate(segments):
+        send = buffers["send"][l % 2][:seg]
+        for i in members[l]:
+            rows, cols = shapes[i]
+            chunk = -(-rows // world)
+            reserved = -(-(chunk * cols) // 8) * 8
+            backend.pack(grad_shards[i], mom_shards[i], cols, reserved, send[offsets[i]:offsets[i] + reserved], stream)
+        if symm is not None:
+            symm.barrier(l % 2)          # every rank has packed bucket l and is done reading bucket l-2
+            ptrs = symm.ptrs(l % 2)
+        else:
+            ptrs = [buffers["send"][l % 2].data_ptr()]
+        if trace is not None:
+            trace.append(("refresh", l))
+        backend.refresh_segments(members[l], ptrs, seg, [offsets[i] for i in members[l]], world, rank,
+                                 [param_shards[i] for i in members[l]], stream)
+    if symm is not None:
+        symm.barrier(0)                  # nobody still reads a buffer that the next step packs into
+    return plan

@@ -228,7 +228,7 @@ def test_bucketed_refresh_needs_a_process_group_for_world_above_one():
 
 
 # ------------------------------------------------------------------- on a GPU
-def _emulate_world(shapes, W, G, M, world, cfg, io, check_mode, bucket_bytes):
+def _emulate_world(shapes, W, G, M, world, cfg, io, check_mode, bucket_bytes, in_place=False):
     """All ranks of `world` one after the other on one device.  Returns full
     (W_new, M_new) as fp64 numpy, shards concatenated."""
     dev = "cuda"
@@ -256,8 +256,12 @@ def _emulate_world(shapes, W, G, M, world, cfg, io, check_mode, bucket_bytes):
         assert not torch.isnan(gathered.float()).any()
         for q in range(world):
             ptrs = [Ws[q][i].t.data_ptr() if Ws[q][i].t.numel() else 0 for i in members]
-            B.prm_refresh_gathered(opt.h, members, gathered.data_ptr(), seg, [offsets[i] for i in members], world, q,
-                                   ptrs, stream)
+            if in_place:        # no gathered copy: every rank's segment is read where it was packed
+                B.prm_refresh_segments(opt.h, members, [x.data_ptr() for x in sends], seg,
+                                       [offsets[i] for i in members], world, q, ptrs, stream)
+            else:
+                B.prm_refresh_gathered(opt.h, members, gathered.data_ptr(), seg, [offsets[i] for i in members], world,
+                                       q, ptrs, stream)
     torch.cuda.synchronize()
     assert opt.status() == B.PRM_OK
     for q in range(world):
@@ -316,6 +320,31 @@ def test_sharded_refresh_tensor_cores_against_oracle_and_across_world_sizes(io):
             # after the bf16 rounding of U, ~1e-5 relative); the bf16 roundings of the recurrence then
             # fall differently, which moves the result by a good part of its own rounding noise.
             assert U.rel_fro(Wn[i], Wu[i]) <= 2e-2, (s, U.rel_fro(Wn[i], Wu[i]))
+
+
+@pytest.mark.gpu
+def test_refresh_segments_reads_every_rank_in_place():
+    shapes = GPU_SHAPES + [(1024, 2560)]
+    cfg = U.oracle_cfg(K=1, beta=0.95, nesterov=True, lr=5e-3, wd=0.01, scale_mode=1)
+    W, G, M = U.make_inputs(shapes, 61, "bf16", grad_std=1e-3, mom_std=1e-3)
+    for world in (1, 3):
+        a = _emulate_world(shapes, W, G, M, world, cfg, "bf16", False, bucket_bytes=2 << 20)
+        b = _emulate_world(shapes, W, G, M, world, cfg, "bf16", False, bucket_bytes=2 << 20, in_place=True)
+        for i in range(len(shapes)):
+            assert np.array_equal(a[0][i], b[0][i]) and np.array_equal(a[1][i], b[1][i])
+
+
+@pytest.mark.gpu
+def test_p2p_exchange_through_symmetric_memory_one_rank():
+    import subprocess
+    import sys
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    worker = os.path.join(os.path.dirname(os.path.abspath(__file__)), "p2p_refresh_worker.py")
+    r = subprocess.run([sys.executable, worker], env=env, capture_output=True, text=True, timeout=600)
+    last = (r.stdout.strip().splitlines() or [""])[-1]
+    if last.startswith("SKIP"):
+        pytest.skip("torch symmetric memory is not usable here: " + last)
+    assert r.returncode == 0 and last == "OK", (r.stdout[-500:], r.stderr[-1500:])
 
 
 @pytest.mark.gpu

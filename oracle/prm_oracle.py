@@ -243,10 +243,11 @@ def adamw_step(p, g, m, v, t, lr=1e-4, beta1=0.9, beta2=0.95, eps=1e-8, wd=0.01)
 # Readings taken here (the paper only says that the Muon matrices are
 # partitioned into communication buckets and that FSDP2 shards dim 0):
 # * rows are split as torch.chunk splits them, chunk = ceil(rows / world);
-# * buckets are filled greedily in the given matrix order, a matrix is never
-#   split, and a bucket is closed when the gathered payload (world segments of
-#   2-byte elements) would exceed the byte cap; every matrix's slot in a
-#   segment is rounded up to 8 elements.  Parity unpinned against the paper
+# * buckets are filled greedily, walking the matrices shape group by shape
+#   group (so that a bucket holds same-shape matrices, which NS5 batches); a
+#   matrix is never split, and a bucket is closed when the gathered payload
+#   (world segments of 2-byte elements) would exceed the byte cap; every
+#   matrix's slot in a segment is rounded up to 8 elements.  Parity unpinned against the paper
 #   (it gives no rule); pinned by the invariants every valid plan must have.
 
 
@@ -259,17 +260,22 @@ def shard_rows(rows, world, rank):
 
 
 def bucket_plan(shapes, world, bucket_bytes):
-    """Communication buckets B_l of Algorithm 2: (bucket_of_mat, offset_in_segment, segment_elems)."""
-    bucket_of_mat, offsets, segments = [], [], []
+    """Communication buckets B_l of Algorithm 2: (bucket_of_mat, offset_in_segment, segment_elems).
+    The matrices are walked shape group by shape group (groups in order of first
+    appearance, given order inside a group)."""
+    groups = group_by_shape(shapes)[0]
+    walk = sorted(range(len(shapes)), key=lambda i: (groups[i], i))
+    bucket_of_mat, offsets, segments = [None] * len(shapes), [None] * len(shapes), []
     seg = 0
-    for (m, n) in shapes:
+    for i in walk:
+        m, n = shapes[i]
         chunk = -(-m // world)
         need = -(-(chunk * n) // 8) * 8
         if seg > 0 and (seg + need) * 2 * world > bucket_bytes:
             segments.append(seg)
             seg = 0
-        bucket_of_mat.append(len(segments))
-        offsets.append(seg)
+        bucket_of_mat[i] = len(segments)
+        offsets[i] = seg
         seg += need
     segments.append(seg)
     return bucket_of_mat, offsets, segments

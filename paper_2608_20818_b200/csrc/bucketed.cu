@@ -21,9 +21,22 @@ extern "C" int prm_bucket_plan(const int64_t* shapes, int n_mats, int world, int
     return PRM_ERR_ARG;
   for (int i = 0; i < n_mats; ++i)
     if (shapes[2 * i] < 1 || shapes[2 * i + 1] < 1) return PRM_ERR_SHAPE;
+  // Walk order: matrices of one shape together (shape groups in order of first appearance, caller
+  // order inside a group), so that a bucket holds matrices that NS5 can batch in one launch.
+  std::vector<int> group(n_mats), order(n_mats);
+  int n_groups = 0;
+  for (int i = 0; i < n_mats; ++i) {
+    int gi = -1;
+    for (int k = 0; k < i && gi < 0; ++k)
+      if (shapes[2 * k] == shapes[2 * i] && shapes[2 * k + 1] == shapes[2 * i + 1]) gi = group[k];
+    group[i] = gi < 0 ? n_groups++ : gi;
+    order[i] = i;
+  }
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return group[a] < group[b]; });
   int bucket = 0;
   int64_t seg = 0;   // elements reserved so far in the current bucket's segment
-  for (int i = 0; i < n_mats; ++i) {
+  for (int k = 0; k < n_mats; ++k) {
+    const int i = order[k];
     // chunk rows of every rank, rounded up to 8 elements so that every matrix starts 16-byte aligned
     const int64_t need = round_up(shard_chunk(shapes[2 * i], world) * shapes[2 * i + 1], 8);
     // gathered payload of the bucket: world segments of bf16

@@ -41,23 +41,29 @@ def test_shard_rows_is_torch_chunk():
 
 def _check_plan(shapes, world, cap, plan):
     bucket_of_mat, offsets, segments = plan
-    assert len(bucket_of_mat) == len(offsets) == len(shapes)
-    assert bucket_of_mat[0] == 0 and all(b1 - b0 in (0, 1) for b0, b1 in zip(bucket_of_mat, bucket_of_mat[1:]))
-    assert len(segments) == bucket_of_mat[-1] + 1
+    n = len(shapes)
+    assert len(bucket_of_mat) == len(offsets) == n
+    # the walk: shape groups in order of first appearance, given order inside a group
+    first = {}
+    for i, sh in enumerate(shapes):
+        first.setdefault(tuple(sh), i)
+    walk = sorted(range(n), key=lambda i: (first[tuple(shapes[i])], i))
+    ids = [bucket_of_mat[i] for i in walk]
+    assert ids[0] == 0 and all(b1 - b0 in (0, 1) for b0, b1 in zip(ids, ids[1:]))
+    assert len(segments) == ids[-1] + 1
+    need = lambda i: -(-(-(-shapes[i][0] // world) * shapes[i][1]) // 8) * 8
     for l, seg in enumerate(segments):
-        members = [i for i, b in enumerate(bucket_of_mat) if b == l]
+        members = [i for i in walk if bucket_of_mat[i] == l]
         assert members, "empty bucket"
         end = 0
-        for i in members:                      # slots in matrix order, disjoint, 16-byte aligned, large enough
-            need = -(-shapes[i][0] // world) * shapes[i][1]
+        for i in members:                      # slots in walk order, disjoint, 16-byte aligned, large enough
             assert offsets[i] == end and offsets[i] % 8 == 0
-            end = offsets[i] + -(-need // 8) * 8
+            end = offsets[i] + need(i)
         assert end == seg
         assert seg * 2 * world <= cap or len(members) == 1
         if l + 1 < len(segments):              # greedy: the next matrix would not have fitted
-            nxt = [i for i, b in enumerate(bucket_of_mat) if b == l + 1][0]
-            need = -(-(-(-shapes[nxt][0] // world) * shapes[nxt][1]) // 8) * 8
-            assert (seg + need) * 2 * world > cap
+            nxt = [i for i in walk if bucket_of_mat[i] == l + 1][0]
+            assert (seg + need(nxt)) * 2 * world > cap
 
 
 def test_bucket_plan_matches_oracle_and_invariants():
@@ -72,9 +78,12 @@ def test_bucket_plan_matches_oracle_and_invariants():
         got = B.prm_bucket_plan(shapes, world, cap)
         assert got == tuple(want) or list(got) == list(want)
         _check_plan(shapes, world, cap, got)
-    # the 9B-class set over 8 ranks in 240 MiB buckets: no bucket holds a whole transformer block
-    b, _, seg = B.prm_bucket_plan([tuple(s) for s in workload(4).shapes], 8, 240 << 20)
+    # the 9B-class set over 8 ranks in 240 MiB buckets: every bucket holds matrices of one shape
+    shapes4 = [tuple(s) for s in workload(4).shapes]
+    b, _, seg = B.prm_bucket_plan(shapes4, 8, 240 << 20)
     assert len(seg) > 42 and max(seg) * 16 <= 240 << 20 + 1
+    mixed = sum(1 for l in range(len(seg)) if len({shapes4[i] for i in range(len(shapes4)) if b[i] == l}) > 1)
+    assert mixed <= 4                          # only where one shape group ends and the next begins
 
 
 def _simulate_pipeline(a, c):

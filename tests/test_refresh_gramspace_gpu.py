@@ -104,3 +104,14 @@ def test_gramspace_is_reproducible_and_close_to_check_mode():
         assert np.array_equal(a[0][i], b[0][i]) and np.array_equal(a[1][i], b[1][i])
         w0 = U.to_np64(W[i])
         assert U.rel_fro((1 - 5e-5) * w0 - a[0][i], (1 - 5e-5) * w0 - c[0][i]) <= TOL
+
+
+@pytest.mark.parametrize("io", ["bf16", "fp32"])
+def test_gramspace_ragged_shapes_and_unaligned_columns(io):
+    # columns not a multiple of 8 take the per-thread final update; fp32 parameters too
+    shapes = [(1030, 2051), (2051, 1030), (1288, 3080), (1025, 2307)]
+    opt = B.PeriodicRowwiseMuon(shapes, 1, io_dtype=io)
+    assert [g["gram_iters"] for g in opt.groups()] == [3, 3, 3, 3]
+    opt.close()
+    errs = _direction_case(shapes, io, False, seed=77)
+    assert max(errs) <= TOL, errs

@@ -6,7 +6,9 @@ The oracle cannot run every matrix of these shape sets, so each case checks
     sampled matrices against the oracle, element by element;
   * the refresh on one whole block (one matrix of every shape): tensor-core
     result against the fp32 check mode for all five shapes, and against the
-    fp64 oracle (all five shapes; the square one only for configuration 5).
+    fp64 oracle (all five shapes; the square one only for configuration 5);
+  * the refresh on every matrix of the set: the Frobenius norm of the
+    direction, which NS5 leaves near sqrt(r).
 Configuration 5 needs 181 GB for its 48 blocks; it runs here with 8 blocks
 (the blocks are identical and independent).
 """
@@ -74,14 +76,21 @@ def _run_config(config_id, blocks, oracle_shapes):
     for i in sample:
         _check_row_step_samples(wl, i, pre[i][0], pre[i][1], grads[i], params[i], moms[i], rng)
 
-    # ---- refresh (t = K).  The sampled block starts from zero parameters, so the step writes
-    # -lr*s*NS5(U) and the bf16 store keeps 2^-9 relative precision on the direction itself.
-    for i in sample:
-        params[i].zero_()
+    # ---- refresh (t = K).  All parameters start from zero, so the step writes -lr*s*NS5(U) and
+    # the bf16 store keeps 2^-9 relative precision on the direction itself.
+    for p in params:
+        p.zero_()
     pre = {i: moms[i].clone() for i in sample}
     opt.step(params, grads, moms, wl.K)
     torch.cuda.synchronize()
     assert opt.status() == B.PRM_OK
+    # Every matrix of the set, whatever sub-batch it was refreshed in: five NS5 iterations leave the
+    # singular values of a well-spread spectrum in a band around one, so ||NS5(U)||_F / sqrt(r) is
+    # of order one (heavy-tailed inputs keep a few small singular values: lower edge 0.3).
+    for i, (m, k) in enumerate(wl.shapes):
+        sc = O.shape_scale(m, k, 1)
+        ratio = float(torch.linalg.norm(params[i].float())) / (wl.lr * sc * min(m, k) ** 0.5)
+        assert 0.3 <= ratio <= 1.2, (i, (m, k), ratio)
     # the same five matrices through the fp32 check mode
     shapes5 = [wl.shapes[i] for i in sample]
     chk = B.PeriodicRowwiseMuon(shapes5, wl.K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma, check_mode=True)

@@ -8,7 +8,9 @@ The oracle cannot run every matrix of these shape sets, so each case checks
     result against the fp32 check mode for all five shapes, and against the
     fp64 oracle (all five shapes; the square one only for configuration 5);
   * the refresh on every matrix of the set: the Frobenius norm of the
-    direction, which NS5 leaves near sqrt(r).
+    direction, which NS5 leaves near sqrt(r);
+  * the row step on every matrix of the set: the norm of every oriented row
+    of the update, which RowNorm fixes at lr*s*gamma.
 Configuration 5 needs 181 GB for its 48 blocks; it runs here with 8 blocks
 (the blocks are identical and independent).
 """
@@ -115,6 +117,18 @@ def _run_config(config_id, blocks, oracle_shapes):
             e_chk = U.rel_fro(U.to_np64(Wc[k]), Wr)
             assert e_fast <= 2e-2, (wl.shapes[i], e_fast)
             assert e_chk <= 4e-3, (wl.shapes[i], e_chk)       # fp32 arithmetic, bf16 store (2^-9)
+    # ---- row step from zero parameters on every matrix of the set: the step writes
+    # -lr*s*gamma*RowNorm(U), so every oriented row (stored row of a wide matrix, stored column of a
+    # tall one) has norm lr*s*gamma, up to the bf16 rounding of its entries.
+    for p in params:
+        p.zero_()
+    opt.step(params, grads, moms, 1)
+    torch.cuda.synchronize()
+    assert opt.status() == B.PRM_OK
+    for i, (m, k) in enumerate(wl.shapes):
+        want = wl.lr * O.shape_scale(m, k, 1) * wl.gamma
+        norms = torch.linalg.vector_norm(params[i].float(), dim=1 if m <= k else 0)
+        assert float((norms / want - 1).abs().max()) <= 2e-3, (i, (m, k))
     opt.close()
     chk.close()
     return out

@@ -378,6 +378,7 @@ def main():
     ap.add_argument("--exchange", default="allgather", choices=["allgather", "p2p"],
                     help="--sharded: NCCL all-gather per bucket, or no collective: the rebuild reads every rank's "
                          "segment in place through symmetric memory (peer loads over NVLink)")
+    ap.add_argument("--no-printed", action="store_true", help="skip the extra refresh steps with the printed NS5")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
@@ -497,6 +498,26 @@ def main():
                "note": "gradients copied every step from pinned host memory (one block's gradients, reused "
                        "for every block) through prm_step_h2d; 2 KB of parameters and the status word read back"}
 
+    # ------------------------------------------ the printed recurrence beside it
+    # The same refresh with all five NS5 iterations evaluated as the paper prints them
+    # (PRM_OPT_NS_GRAM_SPAN = 0), on the same buffers, so that the line carries both figures.
+    printed = None
+    if any(gram_iters.values()) and not args.check_mode and not args.no_printed:
+        opt0 = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
+                                     io_dtype=wl.io_dtype, gram_span=0, device=dev)
+        p0 = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        barrier()
+        for k in range(3):                       # one warm-up refresh, two timed
+            p0[k].record(stream)
+            opt0.step(params, grads, moms, 0)
+        p0[3].record(stream)
+        barrier()
+        assert opt0.status() == B.PRM_OK
+        (ref0,) = max_over_ranks([p0[1].elapsed_time(p0[3]) / 2], dev)
+        printed = {"refresh_ms": ref0}
+        opt0.close()
+        del opt0
+
     if rank != 0:
         if dist:
             td.destroy_process_group()
@@ -573,6 +594,14 @@ def main():
                            "frac": gbs / pk["hbm_gbs"], "traffic": ROW_DRAM_BYTES_PER_ELEMENT * el,
                            "traffic_unit": "DRAM bytes per row step", "kernel": "rowstep_*",
                            "peak_source": "%s copy bandwidth" % pk["source"]}
+    if printed is not None and n_ref:
+        ex0, _ = ns5_flops(wl.shapes)
+        printed["value"] = per_replica_ms((printed["refresh_ms"] + (K - 1) * mean_row) / K if (row_ms or K == 1)
+                                          else printed["refresh_ms"], world)
+        printed["TFLOP/s_exec_whole_refresh"] = ex0 / (printed["refresh_ms"] * 1e-3) / 1e12
+        printed["note"] = ("all five NS5 iterations as printed (PRM_OPT_NS_GRAM_SPAN = 0), two refresh steps timed "
+                           "after the main region; value = amortised ms/step with this refresh and the row step above")
+        out["printed_ns5"] = printed
     out["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
         out["cpu_baseline"] = oracle_sample(wl, K)

@@ -14,8 +14,11 @@
 // 128 rows of P and 128 of the 256 rows of Q in shared memory, and the
 // accumulator rows of its half in its own tensor memory.
 //   warp 0      TMA producer: per stage two 128x64 boxes of P and two of Q
-//               (128 k; cp.async.bulk.tensor, 128-byte swizzle, no multicast);
-//               both CTAs signal the leader's barrier.  Three stages of 64 KB:
+//               (128 k), each operand in ONE copy through a 4-D (k contiguous)
+//               or 5-D (row index contiguous) tensor map whose box spans the
+//               k-blocks and, for the latter, the two 64-wide row blocks
+//               (cp.async.bulk.tensor, 128-byte swizzle, no multicast); both
+//               CTAs signal the leader's barrier.  Three stages of 64 KB:
 //               a stage feeds 8 MMAs, which halves the barrier round trips
 //               per flop against 64-k stages (7 % fewer SM cycles)
 //   warp 1      tcgen05.mma issuer (one lane of the leader CTA); owns the
@@ -153,6 +156,25 @@ __device__ __forceinline__ void tma_load_3d_pair(void* dst, const CUtensorMap* m
   asm volatile(
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(bar_cluster), "r"(x), "r"(y), "r"(z)
+      : "memory");
+}
+// One stage of a K-major operand: kKSub boxes of `rows` x 64 k, fetched as one 4-D box
+// {64 k, rows, kKSub k-blocks, 1}; they land one after the other.
+__device__ __forceinline__ void tma_load_k_stage(void* dst, const CUtensorMap* map, uint32_t bar_cluster, int k0,
+                                                 int row0, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(bar_cluster), "r"(0), "r"(row0), "r"(k0 >> 6), "r"(z)
+      : "memory");
+}
+// One stage of an operand stored with its row index contiguous ([k][n], n fastest): per
+// k-block two adjacent 64 x 64 boxes, fetched as one 5-D box {64 n, 64 k, 2 n-blocks,
+// kKSub k-blocks, 1}.  They land as [k-block][n-block][k][n], the M/N-major operand layout.
+__device__ __forceinline__ void tma_load_t_stage(void* dst, const CUtensorMap* map, uint32_t bar_cluster, int n0,
+                                                 int k0, int z) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+      ::"r"(smem_u32(dst)), "l"((uint64_t)map), "r"(bar_cluster), "r"(0), "r"(0), "r"(n0 >> 6), "r"(k0 >> 6), "r"(z)
       : "memory");
 }
 // shared::cluster address of `p` in the CTA of rank `rank` of this cluster.
@@ -334,27 +356,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           if (rank == 0) mbar_expect_tx(&full[s], 2 * kStageBytes);
           const uint32_t lead_full = lead_full0 + 8u * s;
           const int n0 = c.tj * kBN + (int)rank * (kBN / 2);      // this CTA's 128 rows (columns) of Q
-#pragma unroll
-          for (int kk = 0; kk < kKSub; ++kk) {
-            const int k0 = (kt * kKSub + kk) * kBK;
-            const int kb = k0 / kPad;                             // 256-block of this k-range
-            uint8_t* sp = sa + kk * kBytesA;
-            uint8_t* sq = sa + kKSub * kBytesA + kk * kBytesB;
-            if ((sym_ops & 1) && kb > (c.ti >> 1)) {
-              tma_load_3d_pair(sp, &mapSymP, lead_full, c.ti * kBM, k0, c.b);
-              tma_load_3d_pair(sp + kBytesA / 2, &mapSymP, lead_full, c.ti * kBM + 64, k0, c.b);
-            } else {
-              tma_load_3d_pair(sp, &mapP, lead_full, k0, c.ti * kBM, c.b);
-            }
-            if ((sym_ops & 2) && kb > c.tj) {
-              tma_load_3d_pair(sq, &mapSymQ, lead_full, n0, k0, c.b);
-              tma_load_3d_pair(sq + kBytesB / 2, &mapSymQ, lead_full, n0 + 64, k0, c.b);
-            } else if (!q_mn) {
-              tma_load_3d_pair(sq, &mapQ, lead_full, k0, n0, c.b);
-            } else {
-              tma_load_3d_pair(sq, &mapQ, lead_full, n0, k0, c.b);
-              tma_load_3d_pair(sq + kBytesB / 2, &mapQ, lead_full, n0 + 64, k0, c.b);
-            }
+          const int k0 = kt * kKSub * kBK;
+          const int kb = k0 / kPad;                               // the stage's 128 k lie inside one 256-block
+          uint8_t* sp = sa;
+          uint8_t* sq = sa + kKSub * kBytesA;
+          if ((sym_ops & 1) && kb > (c.ti >> 1)) {
+            tma_load_t_stage(sp, &mapSymP, lead_full, c.ti * kBM, k0, c.b);
+          } else {
+            tma_load_k_stage(sp, &mapP, lead_full, k0, c.ti * kBM, c.b);
+          }
+          if ((sym_ops & 2) && kb > c.tj) {
+            tma_load_t_stage(sq, &mapSymQ, lead_full, n0, k0, c.b);
+          } else if (!q_mn) {
+            tma_load_k_stage(sq, &mapQ, lead_full, k0, n0, c.b);
+          } else {
+            tma_load_t_stage(sq, &mapQ, lead_full, n0, k0, c.b);
           }
         }
       }
@@ -735,6 +751,49 @@ static bool get_map(TcContext* tc, const void* base, int64_t rows, int64_t kdim,
   return true;
 }
 
+// Operand maps: one TMA copy per operand and stage.
+// K-major ([batch][rows][kdim], k contiguous): 4-D {64 k, rows, k-block, batch}, box
+// {64, box_rows, kKSub, 1}.
+static bool get_map_kstage(TcContext* tc, const void* base, int64_t rows, int64_t kdim, int batch, int box_rows,
+                           CUtensorMap* out) {
+  auto key = std::make_tuple(base, rows, kdim, batch, -1000 - box_rows);
+  auto it = tc->cache.find(key);
+  if (it != tc->cache.end()) { *out = it->second; return true; }
+  if (kdim % (kBK * kKSub) != 0) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)kBK, (cuuint64_t)rows, (cuuint64_t)(kdim / kBK), (cuuint64_t)batch};
+  cuuint64_t strides[3] = {(cuuint64_t)kdim * 2, (cuuint64_t)kBK * 2, (cuuint64_t)kdim * (cuuint64_t)rows * 2};
+  cuuint32_t box[4] = {(cuuint32_t)kBK, (cuuint32_t)box_rows, (cuuint32_t)kKSub, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = tc->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
+                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (tc->cache.size() > 4096) tc->cache.clear();
+  tc->cache[key] = *out;
+  return true;
+}
+// Row-index-contiguous ([batch][krows][ncols], n contiguous): 5-D {64 n, 64 k, n-block,
+// k-block, batch}, box {64, 64, 2, kKSub, 1} = 128 n x 128 k in one copy.
+static bool get_map_tstage(TcContext* tc, const void* base, int64_t krows, int64_t ncols, int batch,
+                           CUtensorMap* out) {
+  auto key = std::make_tuple(base, krows, ncols, batch, -5);
+  auto it = tc->cache.find(key);
+  if (it != tc->cache.end()) { *out = it->second; return true; }
+  if (ncols % 128 != 0 || krows % (kBK * kKSub) != 0) return false;
+  cuuint64_t dims[5] = {64, (cuuint64_t)kBK, (cuuint64_t)(ncols / 64), (cuuint64_t)(krows / kBK), (cuuint64_t)batch};
+  cuuint64_t strides[4] = {(cuuint64_t)ncols * 2, 128, (cuuint64_t)ncols * 2 * kBK,
+                           (cuuint64_t)ncols * (cuuint64_t)krows * 2};
+  cuuint32_t box[5] = {64, (cuuint32_t)kBK, 2, (cuuint32_t)kKSub, 1};
+  cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+  CUresult r = tc->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box,
+                          estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  if (tc->cache.size() > 4096) tc->cache.clear();
+  tc->cache[key] = *out;
+  return true;
+}
+
 cudaError_t launch_wait_probe(int* status, uint64_t limit_ns, int* gave_up, cudaStream_t stream) {
   wait_probe_kernel<<<1, 32, 0, stream>>>(status, limit_ns, gave_up);
   return cudaGetLastError();
@@ -764,22 +823,22 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   if (!tc) return cudaErrorInvalidValue;
   if (pb.Mp % kBN != 0 || pb.Np % kBN != 0 || pb.Kp % (kBK * kKSub) != 0) return cudaErrorInvalidValue;
   CUtensorMap mp, mq, maux, maux2, mdst, msp, msq;
-  if (!get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
+  if (!get_map_kstage(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
   if (!pb.q_mn) {
-    if (!get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
+    if (!get_map_kstage(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
   } else {
     // Q stored [batch][Kp][Np]: boxes of 64 k-rows x 64 n
-    if (pb.symmetric || !get_map(tc, pb.Q, pb.Kp, pb.Np, pb.batch, 64, &mq)) return cudaErrorInvalidValue;
+    if (pb.symmetric || !get_map_tstage(tc, pb.Q, pb.Kp, pb.Np, pb.batch, &mq)) return cudaErrorInvalidValue;
   }
   // Epilogue maps (product epilogues only): auxiliary and result slabs of 128
   // rows x 64 columns.
   maux = mp; maux2 = mp; mdst = mp; msp = mp; msq = mp;
   // 64x64 boxes over a symmetric operand, through which its mirrored blocks are read
   if (pb.sym_ops & 1) {
-    if (pb.Mp != pb.Kp || !get_map(tc, pb.P, pb.Mp, pb.Kp, pb.batch, 64, &msp)) return cudaErrorInvalidValue;
+    if (pb.Mp != pb.Kp || !get_map_tstage(tc, pb.P, pb.Mp, pb.Kp, pb.batch, &msp)) return cudaErrorInvalidValue;
   }
   if (pb.sym_ops & 2) {
-    if (pb.Np != pb.Kp || pb.q_mn || !get_map(tc, pb.Q, pb.Np, pb.Kp, pb.batch, 64, &msq)) return cudaErrorInvalidValue;
+    if (pb.Np != pb.Kp || pb.q_mn || !get_map_tstage(tc, pb.Q, pb.Np, pb.Kp, pb.batch, &msq)) return cudaErrorInvalidValue;
   }
   if (ep.aux && (ep.kind == 0 || ep.param_maps)) {
     if (ep.bs_aux != pb.Mp * ep.ld_aux) return cudaErrorInvalidValue;

@@ -36,7 +36,7 @@ NOMINAL_BF16_TFLOPS = 2250.0
 # DRAM traffic of the kernels, from ncu captures of a one-block case of the 9B-class set
 # (profiles/gemm_tc_kernel_dit-9b-class_1block.md, profiles/rowstep_kernels_dit-9b-class_1block.md),
 # scaled to a full launch by the work it processes (traffic grows in proportion to it).
-GEMM_DRAM_BYTES_PER_EXEC_FLOP = 1445.3e6 / (8 * 4096 ** 2 * 12288 + 13 * 4096 ** 3)   # all 18 products of one matrix
+GEMM_DRAM_BYTES_PER_EXEC_FLOP = 1445.6e6 / (8 * 4096 ** 2 * 12288 + 13 * 4096 ** 3)   # all 18 products of one matrix
 ROW_DRAM_BYTES_PER_ELEMENT = 14.0   # wide; the captures never exceed the algorithmic bytes
 
 

@@ -2,6 +2,7 @@
 """Benchmark of the Periodic Row-wise Muon optimizer step on B200.
 
     python bench.py [--gpus N] [--steps S] [--warmup W] [--config 4] [--K 5]
+    python bench.py --gpus N --partition matrices    # whole matrices dealt out to the N ranks
     python bench.py --impl reference ...      # the fp64 CPU oracle on the host cores
 
 One "step" is one prm_step over the whole shape set (a refresh when
@@ -9,11 +10,19 @@ step_idx mod K == 0, a row step otherwise).  The line printed by rank 0 holds
 the amortised optimizer ms/step at K, with per-branch times, the row-step
 GB/s, the NS5 TFLOP/s, a roofline entry for the dominant kernel and the
 oracle's CPU baseline.
+
+With --gpus N > 1 and no launcher around it (WORLD_SIZE unset) the script
+starts its own N ranks through torch.distributed.run on 127.0.0.1; under
+torchrun it is one of the ranks.  N ranks are N independent replicas (weak
+scaling, the default), or share one shape set: by whole matrices
+(--partition matrices: no optimizer collective, NS5 work divided) or by rows
+(--sharded: the paper's Algorithm 2, NS5 replicated).
 """
 
 from __future__ import annotations
 
 import argparse
+import dataclasses
 import json
 import os
 import statistics
@@ -28,16 +37,18 @@ if ROOT not in sys.path:
 
 import torch  # noqa: E402
 
-from paper_2608_20818_b200.workloads import make_grad, make_momentum, make_param, workload  # noqa: E402
+from paper_2608_20818_b200.workloads import (NS_WORKSPACE_BYTES_WHEN_FULL, RESERVE_BYTES, blocks_that_fit,  # noqa: E402
+                                             make_grad, make_momentum, make_param, workload)
 
 METRIC = "amortised optimizer ms/step at K"
 NOMINAL_HBM_GBS = 8000.0       # nominal figure the targets are quoted against
 NOMINAL_BF16_TFLOPS = 2250.0
-# DRAM traffic of the kernels, from ncu captures of a one-block case of the 9B-class set
-# (profiles/gemm_tc_kernel_dit-9b-class_1block.md, profiles/rowstep_kernels_dit-9b-class_1block.md),
-# scaled to a full launch by the work it processes (traffic grows in proportion to it).
+GEMM_CLASSES = ("gram", "poly", "update", "update_final", "gramspace")
+# DRAM traffic of the kernels, from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum) of a
+# one-block case of the 9B-class set, scaled to a full launch by the work it processes (traffic
+# grows in proportion to it).
 GEMM_DRAM_BYTES_PER_EXEC_FLOP = 1445.6e6 / (8 * 4096 ** 2 * 12288 + 13 * 4096 ** 3)   # all 18 products of one matrix
-ROW_DRAM_BYTES_PER_ELEMENT = 14.0   # wide; the captures never exceed the algorithmic bytes
+ROW_DRAM_BYTES_PER_ELEMENT = {"wide": 14.0, "tall": 20.0}   # the tall matrices take two passes over g and m
 
 
 # ----------------------------------------------------------------- accounting
@@ -144,11 +155,10 @@ class ClockSampler:
 def oracle_sample(wl, K, limit_s=20.0):
     """Times the fp64 oracle, as it stands, on a bounded sample of the workload
     and scales it to the whole shape set.  The sample is one matrix of each of
-    the first distinct shapes of the set, as many as are predicted to fit the
-    time limit (always at least one; a square matrix smaller than d x d when
-    even that does not fit); each gets one refresh and one row step.  The
-    refresh is scaled by the paper's flop model 20r^2c+10r^3, the row step by
-    element count."""
+    the cheapest distinct shapes OF THE SET, as many as are predicted to fit the
+    time limit and always at least the cheapest one (never a shape outside the
+    set); each gets one refresh and one row step.  The refresh is scaled by the
+    paper's flop model 20r^2c+10r^3, the row step by element count."""
     import numpy as np
     from oracle import prm_oracle as O
     try:
@@ -176,18 +186,16 @@ def oracle_sample(wl, K, limit_s=20.0):
         if sh not in distinct:
             distinct.append(sh)
     distinct.sort(key=model)
+    # untimed probe (not part of the sample): the host's matmul rate, to predict what fits
     probe = (min(512, min(distinct[0])),) * 2
     one(probe, 0)
-    rate = model(probe) / max(one(probe, 0), 1e-6)           # flop/s of the refresh at probe size
+    rate = model(probe) / max(one(probe, 0), 1e-6)
     sample, predicted = [], 0.0
     for sh in distinct:
         if sample and predicted + model(sh) / rate > limit_s:
             break
         sample.append(sh)
         predicted += model(sh) / rate
-    if len(sample) == 1 and model(sample[0]) / rate > limit_s:   # shrink the only matrix
-        r = max(64, int((limit_s * rate / 30.0) ** (1.0 / 3.0)) // 64 * 64)
-        sample = [(min(r, min(sample[0])),) * 2]
     t_ref = sum(one(sh, 0) for sh in sample)
     t_row = sum(one(sh, 1) for sh in sample) if K > 1 else 0.0
     _, total_model = ns5_flops(wl.shapes)
@@ -198,6 +206,7 @@ def oracle_sample(wl, K, limit_s=20.0):
            f"({t_ref:.2f} s, {t_row:.3f} s), scaled to the shape set by the 20r^2c+10r^3 flop model "
            f"(refresh) and by element count (row step)")
     return {"value": amort, "unit": "ms/step", "cores": cores, "kind": "oracle", "sample": txt,
+            "shapes_sampled": "%d of %d distinct shapes of the set" % (len(sample), len(distinct)),
             "refresh_ms": ref_ms, "row_step_ms": row_ms}
 
 
@@ -355,7 +364,7 @@ def run_sharded(args, wl, K, rank, local_rank, world, dev):
     print(json.dumps(out))
 
 
-def main():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
@@ -371,6 +380,9 @@ def main():
     ap.add_argument("--ns5-schedule", type=int, default=2, choices=[0, 1, 2],
                     help="PRM_OPT_NS_GRAM_SPAN: 0 printed recurrence, 1 first three iterations in Gram space, "
                          "2 (library default) also the last Gram matrix from the one before it")
+    ap.add_argument("--partition", default="replicas", choices=["replicas", "matrices"],
+                    help="N > 1: independent replicas (weak scaling), or one shape set whose matrices are dealt "
+                         "out to the ranks by prm_partition_matrices (strong scaling, no optimizer collective)")
     ap.add_argument("--sharded", action="store_true",
                     help="the paper's distributed execution over the N ranks (rows sharded, bucketed all-gather "
                          "refresh, sharded tall RowNorm) instead of N independent replicas")
@@ -381,8 +393,87 @@ def main():
     ap.add_argument("--no-printed", action="store_true", help="skip the extra refresh steps with the printed NS5")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
+    ap.add_argument("--dry-run", action="store_true",
+                    help="launcher and partition logic only, on CPU ranks (gloo): every rank plans its matrix list "
+                         "and runs a stub step; no CUDA work, no timing claim")
+    return ap.parse_args(argv)
 
+
+def launch_ranks(n, argv):
+    """Start n ranks of this script on this node through torch.distributed.run
+    (rendezvous on 127.0.0.1) and pass their output through."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--standalone", "--nnodes=1", f"--nproc-per-node={n}",
+           "--local-addr", "127.0.0.1", os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def rank_matrix_list(shapes, world, rank):
+    """(indices into `shapes` owned by `rank`, NS5 cost per rank in flop) under
+    the whole-matrix partition (prm_partition_matrices, a host-only call)."""
+    from paper_2608_20818_b200 import binding as B
+    owner, cost = B.prm_partition_matrices([tuple(s) for s in shapes], world)
+    return [i for i, q in enumerate(owner) if q == rank], cost
+
+
+def run_dry(args, wl, K, rank, world):
+    """The N-rank plumbing without a GPU: each rank takes its matrix list, runs
+    a stub step over it, and rank 0 gathers the lists and prints the line."""
+    import torch.distributed as td
+    dist = world > 1
+    if dist:
+        td.init_process_group("gloo")
+    if args.partition == "matrices":
+        mine, cost = rank_matrix_list(wl.shapes, world, rank)
+    else:
+        mine, cost = list(range(len(wl.shapes))), [float(ns5_flops(wl.shapes)[0])] * world
+    t0 = time.perf_counter()
+    touched = sum(wl.shapes[i][0] * wl.shapes[i][1] for i in mine)      # the stub step: walk the list
+    stub_ms = (time.perf_counter() - t0) * 1e3
+    (stub_ms,) = max_over_ranks([stub_ms])
+    lists = [None] * world
+    if dist:
+        td.all_gather_object(lists, mine)
+    else:
+        lists = [mine]
+    if rank == 0:
+        print(json.dumps({"dry_run": True, "n_gpus": world, "partition": args.partition,
+                          "scaling": "strong" if args.partition == "matrices" else "weak",
+                          "config": {"workload": wl.name, "K": K, "matrices": len(wl.shapes)},
+                          "matrix_lists": lists, "ns5_flop_per_rank": cost, "elements_rank0": touched,
+                          "stub_ms": stub_ms}))
+    if dist:
+        td.barrier()
+        td.destroy_process_group()
+
+
+def main(argv=None):
+    args = parse_args(argv)
+    raw_argv = list(sys.argv[1:] if argv is None else argv)
+    if args.gpus < 1:
+        raise SystemExit("--gpus must be >= 1")
+    launched = "WORLD_SIZE" in os.environ
+    if args.gpus > 1 and not launched:
+        # no launcher around this process: start the N ranks ourselves (the reference arm too:
+        # its rank 0 prints, the others leave at once)
+        raise SystemExit(launch_ranks(args.gpus, raw_argv))
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} does not match WORLD_SIZE={world}")
+
+    full = workload(args.config)
+    mem = None
+    if args.impl == "prm" and not args.dry_run:
+        torch.cuda.set_device(local_rank)
+        free_b, total_b = torch.cuda.mem_get_info()
+        mem = {"free_gib": round(free_b / 2 ** 30, 2), "total_gib": round(total_b / 2 ** 30, 2)}
+        if args.blocks is None and full.blocks and args.partition == "replicas" and not args.sharded:
+            # the largest block count of the configuration that this device holds (all of them on a
+            # B200 for configurations 2-5 when its memory is free)
+            args.blocks = blocks_that_fit(args.config, free_b)
+            mem["blocks_that_fit"] = args.blocks
     wl = workload(args.config, args.blocks)
     K = args.K or wl.K
     if args.steps is None:
@@ -392,14 +483,13 @@ def main():
     if args.impl == "reference":
         run_reference(args, wl, K)
         return
+    if args.dry_run:
+        run_dry(args, wl, K, rank, world)
+        return
 
     from paper_2608_20818_b200 import binding as B
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
     dist = world > 1
-    torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     if dist:
         import torch.distributed as td
@@ -411,18 +501,44 @@ def main():
             td.destroy_process_group()
         return
 
+    # ------------------------------------------------- this rank's matrices
+    set_shapes = wl.shapes                       # the shape set the job as a whole steps
+    part_cost = None
+    if args.partition == "matrices" and world > 1:
+        mine, part_cost = rank_matrix_list(wl.shapes, world, rank)
+        wl = dataclasses.replace(wl, shapes=tuple(wl.shapes[i] for i in mine))
     n = len(wl.shapes)
     io_bytes = 4 if wl.io_dtype == "fp32" else 2
+    resident = elements(wl.shapes) * (2 * io_bytes + 4)
+    nearly_full = mem is not None and resident > 0.8 * mem["free_gib"] * 2 ** 30
+    ns_cap = NS_WORKSPACE_BYTES_WHEN_FULL if nearly_full else None
     opt = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
-                                io_dtype=wl.io_dtype, check_mode=args.check_mode, gram_span=0 if args.printed_ns5 else args.ns5_schedule,
-                                device=dev)
+                                io_dtype=wl.io_dtype, check_mode=args.check_mode,
+                                gram_span=0 if args.printed_ns5 else args.ns5_schedule,
+                                ns_workspace_bytes=ns_cap, device=dev)
     gram_iters = {(g["rows"], g["cols"]): g["gram_iters"] for g in opt.groups()}
     exec_flop = {(g["rows"], g["cols"]): g["ns5_flop"] for g in opt.groups()}
-    params = [make_param(wl, i, dev) for i in range(n)]
-    moms = [make_momentum(wl, i, dev) for i in range(n)]
-    # One gradient set per matrix kind and step parity keeps generation cheap;
-    # every matrix still owns its own gradient buffer in HBM.
-    grads = [make_grad(wl, i, 0, dev) for i in range(n)]
+    params, moms = [], []
+    for i in range(n):
+        params.append(make_param(wl, i, dev))
+        moms.append(make_momentum(wl, i, dev))
+        if i % 5 == 4:
+            torch.cuda.empty_cache()             # the generators' fp32 temporaries
+    # Gradients: every matrix owns its gradient buffer in HBM.  Two full sets (seeded for step 0 and
+    # step 1) alternate from step to step where a second set fits beside the shape set; otherwise
+    # one set is reused (timing does not depend on the values).
+    free_now = torch.cuda.mem_get_info()[0]
+    grad_bytes = elements(wl.shapes) * io_bytes
+    n_sets = 2 if free_now - 2 * grad_bytes > RESERVE_BYTES else 1
+    grad_sets = []
+    for sset in range(n_sets):
+        gs = []
+        for i in range(n):
+            gs.append(make_grad(wl, i, sset, dev))
+            if i % 5 == 4:
+                torch.cuda.empty_cache()
+        grad_sets.append(gs)
+    grads = grad_sets[0]
     torch.cuda.synchronize()
 
     stream = torch.cuda.current_stream(dev)
@@ -437,7 +553,7 @@ def main():
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
-        opt.step(params, grads, moms, step_idx)
+        opt.step(params, grad_sets[step_idx % n_sets], moms, step_idx)
         step_idx += 1
     barrier()
     assert opt.status() == B.PRM_OK, "device status after warm-up"
@@ -451,7 +567,7 @@ def main():
     ev[0].record(stream)
     for k in range(args.steps):
         kinds.append(opt.plan(step_idx)[0])
-        opt.step(params, grads, moms, step_idx)
+        opt.step(params, grad_sets[step_idx % n_sets], moms, step_idx)
         ev[k + 1].record(stream)
         step_idx += 1
     barrier()
@@ -471,11 +587,14 @@ def main():
     # ---------------------------------------------------------- e2e (host grads)
     e2e = None
     if not args.no_e2e:
-        block = 5 if wl.config_id != 1 else 1
-        host = [torch.empty(wl.shapes[i], dtype=grads[i].dtype).pin_memory() for i in range(min(block, n))]
-        for i, h in enumerate(host):
-            h.copy_(grads[i])
-        grads_host = [host[i % block] for i in range(n)]
+        # pinned host gradients: one matrix of each shape stands for every matrix of that shape
+        by_shape = {}
+        for i in range(n):
+            if tuple(wl.shapes[i]) not in by_shape:
+                hbuf = torch.empty(wl.shapes[i], dtype=grads[i].dtype).pin_memory()
+                hbuf.copy_(grads[i])
+                by_shape[tuple(wl.shapes[i])] = hbuf
+        grads_host = [by_shape[tuple(wl.shapes[i])] for i in range(n)]
         readback = torch.empty(1024, dtype=params[0].dtype).pin_memory()
         h2d = sum(m * nn for (m, nn) in wl.shapes) * io_bytes
         d2h = readback.numel() * readback.element_size() + 4
@@ -493,10 +612,12 @@ def main():
         t1.record(stream)
         barrier()
         (e_ms,) = max_over_ranks([t0.elapsed_time(t1) / e_steps], dev)
-        e2e = {"value": per_replica_ms(e_ms, world), "unit": "ms/step", "h2d_bytes_per_step": h2d,
+        weak = args.partition == "replicas"
+        e2e = {"value": per_replica_ms(e_ms, world) if weak else e_ms, "unit": "ms/step", "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": d2h,
-               "note": "gradients copied every step from pinned host memory (one block's gradients, reused "
-                       "for every block) through prm_step_h2d; 2 KB of parameters and the status word read back"}
+               "note": "gradients copied every step from pinned host memory (one matrix of each shape, reused "
+                       "for every matrix of that shape) through prm_step_h2d; 2 KB of parameters and the status "
+                       "word read back: this figure is the host link (PCIe), not the kernels"}
 
     # ------------------------------------------ the printed recurrence beside it
     # The same refresh with all five NS5 iterations evaluated as the paper prints them
@@ -504,17 +625,21 @@ def main():
     printed = None
     if any(gram_iters.values()) and not args.check_mode and not args.no_printed:
         opt0 = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
-                                     io_dtype=wl.io_dtype, gram_span=0, device=dev)
+                                     io_dtype=wl.io_dtype, gram_span=0, ns_workspace_bytes=ns_cap, device=dev)
         p0 = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
         barrier()
         for k in range(3):                       # one warm-up refresh, two timed
+            if k == 1:
+                opt0.profile(True)
             p0[k].record(stream)
             opt0.step(params, grads, moms, 0)
         p0[3].record(stream)
         barrier()
+        prof0 = opt0.profile_read()
         assert opt0.status() == B.PRM_OK
         (ref0,) = max_over_ranks([p0[1].elapsed_time(p0[3]) / 2], dev)
-        printed = {"refresh_ms": ref0}
+        printed = {"refresh_ms": ref0,
+                   "gemm_ms_per_refresh": sum(prof0[k][0] for k in GEMM_CLASSES) / 2}
         opt0.close()
         del opt0
 
@@ -524,30 +649,41 @@ def main():
         return
 
     pk = peaks()
+    weak = args.partition == "replicas"
     amort = (mean_ref + (K - 1) * mean_row) / K if (ref_ms and (row_ms or K == 1)) else total_ms / args.steps
     n_ref, n_row = len(ref_ms), len(row_ms)
     ex, mo = ns5_flops(wl.shapes, exec_flop)
     ex_printed, _ = ns5_flops(wl.shapes)
     el = elements(wl.shapes)
+    el_tall = elements([sh for sh in wl.shapes if sh[0] > sh[1]])
     row_bytes = el * (3 * io_bytes + 8)   # g and p read, p write (I/O dtype), m read and write (fp32)
-    gemm_classes = ("gram", "poly", "update", "update_final", "gramspace")
-    gemm_ms = sum(prof[k][0] for k in gemm_classes)
-    gemm_launches = sum(prof[k][1] for k in gemm_classes)
+    gemm_ms = sum(prof[k][0] for k in GEMM_CLASSES)
+    gemm_launches = sum(prof[k][1] for k in GEMM_CLASSES)
     row_kernel_ms = prof["row_wide"][0] + prof["row_tall"][0]
+    if world == 1:
+        parallelism = "one GPU"
+    elif weak:
+        parallelism = "%d independent replicas" % world
+    else:
+        parallelism = "whole matrices dealt out to %d ranks (prm_partition_matrices), no optimizer collective" % world
     out = {
-        "metric": METRIC, "value": per_replica_ms(amort, world), "unit": "ms/step", "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": False,
-        "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": per_replica_ms(amort, world) if weak else amort, "unit": "ms/step", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": False,
+        "scaling": "weak" if weak else "strong", "vs_baseline": None,
         "dtype": "f32" if args.check_mode else "bf16", "data": "synthetic",
-        "config": {"workload": wl.name, "K": K, "matrices": n, "blocks": wl.blocks, "d": wl.d,
-                   "elements": el, "io_dtype": wl.io_dtype, "momentum_dtype": "fp32",
+        "config": {"workload": wl.name, "K": K, "matrices": len(set_shapes), "blocks": wl.blocks,
+                   "blocks_stated": full.blocks, "d": wl.d,
+                   "elements": elements(set_shapes), "io_dtype": wl.io_dtype, "momentum_dtype": "fp32",
                    "ns5": "fp32 check mode" if args.check_mode else "bf16 tcgen05",
                    "ns5_schedule": ("five iterations as printed" if not any(gram_iters.values()) else
                                     "PRM_OPT_NS_GRAM_SPAN=%d: iterations 1-3 in Gram space for %d of %d matrices%s" % (
                                         args.ns5_schedule, sum(1 for sh in wl.shapes if gram_iters.get(tuple(sh), 0)), n,
                                         ", last Gram matrix from the previous one where c > 2r"
                                         if args.ns5_schedule == 2 else "")),
-                   "replicas": world, "l2": "inputs larger than L2 (working set %.1f GB)" % (el * 8 / 1e9),
+                   "parallelism": parallelism, "matrices_rank0": n,
+                   "device_memory": mem, "ns_workspace_cap_bytes": ns_cap,
+                   "gradient_sets": n_sets,
+                   "l2": "inputs larger than L2 (working set %.1f GB)" % (el * 8 / 1e9),
                    "first_timed_step_index": t_first + args.warmup},
         "refresh_ms": mean_ref if n_ref else None, "row_step_ms": mean_row if n_row else None,
         "refresh_steps_timed": n_ref, "row_steps_timed": n_row,
@@ -556,23 +692,30 @@ def main():
         # device time per kernel class over the whole timed region (CUDA events inside the library)
         "kernel_classes": {k: {"ms": round(v[0], 3), "launches": v[1]} for k, v in prof.items()},
     }
+    if part_cost is not None:
+        out["config"]["ns5_flop_per_rank"] = part_cost
     if n_row:
         gbs = row_bytes / (mean_row * 1e-3) / 1e9
         out["row_step"] = {"GB/s": gbs, "bytes_per_element": 3 * io_bytes + 8,
                            "frac_of_measured_peak": gbs / pk["hbm_gbs"], "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
-                           "kernel_ms_per_step": row_kernel_ms / n_row}
+                           "kernel_ms_per_step": row_kernel_ms / n_row,
+                           "wide_ms_per_step": prof["row_wide"][0] / n_row, "tall_ms_per_step": prof["row_tall"][0] / n_row,
+                           "tall_GB/s": (el_tall * (3 * io_bytes + 8) / (prof["row_tall"][0] / n_row * 1e-3) / 1e9
+                                         if prof["row_tall"][0] > 0 else None)}
     if n_ref and gemm_ms > 0:
         tf_exec = ex * n_ref / (gemm_ms * 1e-3) / 1e12
-        out["ns5"] = {"TFLOP/s_exec": tf_exec, "TFLOP/s_model": mo * n_ref / (gemm_ms * 1e-3) / 1e12,
-                      # the printed recurrence's symmetric count over the same time: what a kernel that ran
-                      # all five iterations on X would have to sustain to be as fast
-                      "TFLOP/s_printed_equivalent": ex_printed * n_ref / (gemm_ms * 1e-3) / 1e12,
+        out["ns5"] = {"TFLOP/s_exec": tf_exec,
                       "exec_flop_per_refresh": ex, "printed_flop_per_refresh": ex_printed,
                       "TFLOP/s_exec_whole_refresh": ex / (mean_ref * 1e-3) / 1e12,
                       "frac_of_measured_burst": tf_exec / pk["bf16_tflops"],
                       "frac_of_measured_sustained": tf_exec / pk["bf16_tflops_sustained"],
                       "frac_of_nominal_2250": tf_exec / NOMINAL_BF16_TFLOPS,
-                      "gemm_ms_per_refresh": gemm_ms / n_ref, "prepass_ms_per_refresh": prof["prepass"][0] / n_ref}
+                      "gemm_ms_per_refresh": gemm_ms / n_ref, "prepass_ms_per_refresh": prof["prepass"][0] / n_ref,
+                      # flop counts the kernels do NOT execute, over the same time: for comparison with the
+                      # paper's accounting only
+                      "model_equivalents": {"not_a_rate": True,
+                                            "paper_model_20r2c_10r3": mo * n_ref / (gemm_ms * 1e-3) / 1e12,
+                                            "printed_recurrence_symmetric": ex_printed * n_ref / (gemm_ms * 1e-3) / 1e12}}
         if args.check_mode:
             # fp32 FMA path: bounded by CUDA-core arithmetic, not by tensor cores
             peak = 148 * 128 * 2 * 1.965e9 / 1e12
@@ -590,15 +733,21 @@ def main():
                                "peak_source": "%s sustained bf16 matmul" % pk["source"]}
     elif n_row:
         gbs = row_bytes / (row_kernel_ms / n_row * 1e-3) / 1e9
+        traffic = (ROW_DRAM_BYTES_PER_ELEMENT["wide"] * (el - el_tall) + ROW_DRAM_BYTES_PER_ELEMENT["tall"] * el_tall)
         out["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                           "frac": gbs / pk["hbm_gbs"], "traffic": ROW_DRAM_BYTES_PER_ELEMENT * el,
+                           "frac": gbs / pk["hbm_gbs"], "traffic": traffic,
                            "traffic_unit": "DRAM bytes per row step", "kernel": "rowstep_*",
                            "peak_source": "%s copy bandwidth" % pk["source"]}
     if printed is not None and n_ref:
         ex0, _ = ns5_flops(wl.shapes)
-        printed["value"] = per_replica_ms((printed["refresh_ms"] + (K - 1) * mean_row) / K if (row_ms or K == 1)
-                                          else printed["refresh_ms"], world)
+        v0 = (printed["refresh_ms"] + (K - 1) * mean_row) / K if (row_ms or K == 1) else printed["refresh_ms"]
+        printed["value"] = per_replica_ms(v0, world) if weak else v0
         printed["TFLOP/s_exec_whole_refresh"] = ex0 / (printed["refresh_ms"] * 1e-3) / 1e12
+        if printed["gemm_ms_per_refresh"] > 0:
+            printed["TFLOP/s_exec"] = ex0 / (printed["gemm_ms_per_refresh"] * 1e-3) / 1e12
+            if "roofline" in out and out["roofline"]["bound"] == "tensor":
+                # the same kernel running the recurrence exactly as printed, against the same peak
+                out["roofline"]["frac_printed_schedule"] = printed["TFLOP/s_exec"] / out["roofline"]["peak"]
         printed["note"] = ("all five NS5 iterations as printed (PRM_OPT_NS_GRAM_SPAN = 0), two refresh steps timed "
                            "after the main region; value = amortised ms/step with this refresh and the row step above")
         out["printed_ns5"] = printed

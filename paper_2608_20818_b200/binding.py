@@ -230,7 +230,19 @@ def prm_rowstep_tall_noalloc(param, grad, momentum, *, beta, nesterov, lr, wd, g
     memory (no workspace, no handle): the scratch sits in a fixed array inside
     the library.  Tensors are updated in place; see include/prm.h for the size
     limit and the sharing rules of that array."""
+    if len(param.shape) != 2:
+        raise ValueError("param must be a 2-D matrix")
     rows, cols = param.shape
+    if param.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("param must be float32 or bfloat16")
+    if grad.dtype != param.dtype or momentum.dtype != torch.float32:
+        raise TypeError(f"dtypes must be {param.dtype} (param, grad) and float32 (momentum)")
+    if tuple(grad.shape) != tuple(param.shape) or tuple(momentum.shape) != tuple(param.shape):
+        raise ValueError("param, grad and momentum must have the same shape")
+    if not (param.is_contiguous() and grad.is_contiguous() and momentum.is_contiguous()):
+        raise ValueError("param, grad and momentum must be contiguous")
+    if param.device.type != "cuda" or grad.device != param.device or momentum.device != param.device:
+        raise ValueError("param, grad and momentum must sit on the same CUDA device")
     io_fp32 = 1 if param.dtype == torch.float32 else 0
     s = (stream or torch.cuda.current_stream(param.device)).cuda_stream
     buf = ctypes.create_string_buffer(256)

@@ -99,7 +99,6 @@ static float shape_scale(int mode, int64_t rows, int64_t cols) {
 }
 
 static void compute_layout(prm_ctx* c) {
-  const size_t e = c->check_mode ? 4 : 2;
   size_t off = 0;
   c->off_status = off; off += 256;
   c->off_tables = off; off = align_up(off + (size_t)3 * c->n_mats * sizeof(void*), 256);
@@ -115,7 +114,9 @@ static void compute_layout(prm_ctx* c) {
     // Gram-space iterations trade 6 r^2 (c - r) flop for six r^3 products: worth it
     // from c = 1.5 r on; below 1024 rows the time is noise and the bf16 rounding of the
     // small r x r matrices averages less well, so those stay on the printed recurrence.
-    g.gram_iters = (!c->check_mode && c->gram_span && g.rp >= 1024 && 2 * g.cp >= 3 * g.rp) ? kGramIters : 0;
+    g.ns_fp32 = (c->check_mode || g.r < kTinyRows) ? 1 : 0;
+    const size_t e = g.ns_fp32 ? 4 : 2;
+    g.gram_iters = (!g.ns_fp32 && c->gram_span && g.rp >= 1024 && 2 * g.cp >= 3 * g.rp) ? kGramIters : 0;
     // Mode 2: beyond c = 2r the Gram matrix of the last iteration is also cheaper from the one
     // before it (A_4 = P_3 A_3 P_3, two r^3 products) than from X_4 (one r^2 c product).
     g.last_gram_rec = (g.gram_iters && c->gram_span >= 2 && g.cp > 2 * g.rp) ? 1 : 0;
@@ -290,7 +291,7 @@ struct NsFinal {
 // Returns the index (0 or 1) of the X buffer that holds X_5 when fin is null.
 static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFinal* fin, int* x_out,
                                 cudaStream_t stream) {
-  const size_t e = c->check_mode ? 4 : 2;
+  const size_t e = g.ns_fp32 ? 4 : 2;
   const int64_t rc = g.rp * g.cp, rr = g.rp * g.rp;
   float* alpha = (float*)(c->ws + c->off_alpha);
   int* status = (int*)(c->ws + c->off_status);
@@ -303,8 +304,8 @@ static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFina
   cudaError_t ce;
   auto gemm = [&](const GemmProblem& pb, const Epilogue& ep, int cls) -> cudaError_t {
     ProfScope ps(c, cls, stream);
-    return c->check_mode ? launch_gemm_simt(pb, ep, stream, &c->launches)
-                         : launch_gemm_tc(c->tc, pb, ep, status, stream, &c->launches);
+    return g.ns_fp32 ? launch_gemm_simt(pb, ep, stream, &c->launches)
+                     : launch_gemm_tc(c->tc, pb, ep, status, stream, &c->launches);
   };
   int cur = 0, it0 = 0;
   ce = cudaSuccess;
@@ -414,7 +415,7 @@ static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFina
       eu.rows = (int)g.rows; eu.cols = (int)g.cols; eu.tall = g.tall ? 1 : 0;
       eu.io_fp32 = c->io_fp32; eu.decay = fin->decay; eu.lr_s = fin->lr_s;
       // bf16 parameters with 16-byte aligned rows are updated through TMA-staged tiles.
-      if (!c->check_mode && !c->io_fp32 && g.cols % 8 == 0) eu.param_maps = c->ws + c->off_pmaps;
+      if (!g.ns_fp32 && !c->io_fp32 && g.cols % 8 == 0) eu.param_maps = c->ws + c->off_pmaps;
     }
     if ((ce = gemm(pu, eu, it + 1 < kNsIters ? PRM_PROF_UPDATE : PRM_PROF_UPDATE_FINAL)) != cudaSuccess) break;
     cur ^= 1;
@@ -433,7 +434,7 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
     cudaError_t ce;
     {
       ProfScope ps(c, PRM_PROF_PREPASS, stream);
-      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, c->check_mode, c->ws + c->off_ns, fro, alpha, stream,
+      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, g.ns_fp32, c->ws + c->off_ns, fro, alpha, stream,
                              &c->launches);
     }
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("pre-pass: ") + cudaGetErrorString(ce));
@@ -481,11 +482,11 @@ extern "C" int prm_refresh_segments(prm_ctx* c, const int* mats, int n, const vo
   }
   float* fro = (float*)(c->ws + c->off_fro);
   float* alpha = (float*)(c->ws + c->off_alpha);
-  const size_t e = c->check_mode ? 4 : 2;
   std::vector<int64_t> offs;
   std::vector<void*> shards;
   for (size_t gi = 0; gi < c->groups.size(); ++gi) {
     const Group& g = c->groups[gi];
+    const size_t e = g.ns_fp32 ? 4 : 2;
     offs.clear();
     shards.clear();
     for (int k = 0; k < n; ++k)
@@ -502,7 +503,7 @@ extern "C" int prm_refresh_segments(prm_ctx* c, const int* mats, int n, const vo
       {
         ProfScope ps(c, PRM_PROF_PREPASS, stream);
         ce = launch_ns_gather_prepass(segs, vec_ok, shard_chunk(g.rows, world), offs.data() + done, g, nb,
-                                      c->eps_ns, c->check_mode, c->ws + c->off_ns, fro, alpha, stream, &c->launches);
+                                      c->eps_ns, g.ns_fp32, c->ws + c->off_ns, fro, alpha, stream, &c->launches);
       }
       if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("gathered pre-pass: ") + cudaGetErrorString(ce));
       int xi = 0;
@@ -511,7 +512,7 @@ extern "C" int prm_refresh_segments(prm_ctx* c, const int* mats, int n, const vo
       {
         ProfScope ps(c, PRM_PROF_UPDATE_FINAL, stream);
         const char* X5 = c->ws + c->off_ns + (size_t)xi * e * (size_t)(g.rp * g.cp) * nb;
-        ce = launch_ns_slice_update(X5, c->check_mode, g, nb, shards.data() + done, row_start, rows_local, c->io_fp32,
+        ce = launch_ns_slice_update(X5, g.ns_fp32, g, nb, shards.data() + done, row_start, rows_local, c->io_fp32,
                                     decay, lr_s, stream, &c->launches);
       }
       if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("slice update: ") + cudaGetErrorString(ce));
@@ -563,7 +564,7 @@ static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
     if (!c->check_mode && !c->io_fp32) {
       for (int i = 0; i < n; ++i) {
         const Group& g = c->groups[c->group_of_mat[i]];
-        if (g.cols % 8 != 0) continue;
+        if (g.cols % 8 != 0 || g.ns_fp32) continue;
         if (!tc_encode_param_map(c->tc, params[i], g.rows, g.cols, g.tall ? 1 : 0,
                                  c->host_pmaps.data() + (size_t)128 * c->slot_of_mat[i]))
           return fail(c, PRM_ERR_CUDA, "cannot encode a tensor map over a parameter matrix");

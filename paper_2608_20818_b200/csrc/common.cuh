@@ -26,6 +26,14 @@ constexpr int kGramIters = 3;   // leading iterations that can run on the r x r 
 // dimensions; the padding is zero and stays zero through the recurrence.
 constexpr int kPad = 256;
 
+// Matrices with fewer oriented rows than this are refreshed in fp32 on CUDA
+// cores even outside the check mode.  With so few rows the bf16 rounding of
+// the r x r matrices does not average out: emulating bf16 storage with fp32
+// accumulation on the CPU gives relative errors of the direction up to 6e-2
+// at 5 rows and 2-3e-2 at 32 rows, against 1.2e-2 from 64 rows on.  The work
+// is a single 256-row tile per product.
+constexpr int kTinyRows = 64;
+
 // Tall row-step: rows per column-partial block.
 constexpr int kTallRows = 128;
 // Tall row-step and pre-pass: columns per CTA.
@@ -158,6 +166,7 @@ struct Group {
   int ns_batch = 1;             // matrices refreshed per sub-batch
   int gram_iters = 0;           // leading NS5 iterations run in Gram space (0 or kGramIters)
   int last_gram_rec = 0;        // 1: the last iteration's Gram matrix comes from the previous one's
+  int ns_fp32 = 0;              // 1: NS5 of this group runs in fp32 on CUDA cores (check mode, or a tiny matrix)
   size_t tall_scratch_off = 0;  // byte offset of column partials (tall groups)
   size_t tall_nu_off = 0;       // byte offset of column norms (tall groups)
 };

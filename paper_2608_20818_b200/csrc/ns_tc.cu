@@ -200,6 +200,13 @@ __device__ __forceinline__ void tma_store_3d(const void* src, const CUtensorMap*
                ::"l"((uint64_t)map), "r"(smem_u32(src)), "r"(x), "r"(y), "r"(z)
                : "memory");
 }
+// The parameter tensor maps live in global memory and are rewritten by a host
+// copy whenever the caller moves its parameters.  An SM may still hold the
+// descriptor it fetched from that address in an earlier launch; the acquire
+// fence on the tensor-map proxy makes the next use fetch it again.
+__device__ __forceinline__ void tensormap_acquire(const CUtensorMap* map) {
+  asm volatile("fence.proxy.tensormap::generic.acquire.sys [%0], 128;" ::"l"((uint64_t)map) : "memory");
+}
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
@@ -442,6 +449,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
       int n_my_tiles = 0;
       for (int t = blockIdx.x; t < total_tiles; t += gridDim.x) ++n_my_tiles;
       const uint32_t n_slabs = (uint32_t)n_my_tiles * kSlabs;
+      int fenced_b = -1;                 // matrix whose parameter map has been acquired
       auto prepare = [&](uint32_t g) {
         const int bsel = g % kEpiBufs;
         if (has_aux || fin) {
@@ -455,6 +463,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
             // Parameter tile into the second slab: as stored (wide), or the
             // transposed region in two 64x64 boxes (tall).  Out-of-range parts read as zero.
             const CUtensorMap* pm = pmaps + ep.first + c.b;
+            if (c.b != fenced_b) { tensormap_acquire(pm); fenced_b = c.b; }
             if (!ep.tall) {
               tma_load_2d(buf + kSlabBytes, pm, &eready[bsel], j0, c.ti * kBM);
             } else {

@@ -71,6 +71,32 @@ def workload(config_id: int, blocks: int | None = None) -> Workload:
                     shapes=tuple(dit_shapes(d, nb)))
 
 
+# Memory sizing of a shape set (no optimizer arithmetic): what the caller keeps
+# resident per transformer block, and how many blocks a GPU can hold.
+RESERVE_BYTES = 8 << 30          # workspace of the optimizer, the caching allocator's slack, test scratch
+NS_WORKSPACE_BYTES_WHEN_FULL = 2 << 30   # NS5 workspace cap used when the set nearly fills the GPU
+
+
+def block_resident_bytes(d: int, io_dtype: str = "bf16") -> int:
+    """Bytes of parameters, gradients (I/O dtype) and fp32 momentum of one block (18 d^2 elements)."""
+    io = 4 if io_dtype == "fp32" else 2
+    return 18 * d * d * (2 * io + 4)
+
+
+def blocks_that_fit(config_id: int, free_bytes: int, reserve_bytes: int = RESERVE_BYTES) -> int:
+    """The largest block count of configuration `config_id` (at most its stated
+    count) whose resident tensors fit `free_bytes` of device memory with
+    `reserve_bytes` left over.  The test at full size and the benchmark both
+    call this with the figure torch.cuda.mem_get_info() reports, so they run the
+    same subset.  Blocks are identical and independent: time is linear in their
+    number."""
+    wl = workload(config_id)
+    if wl.blocks == 0:
+        return 0
+    per = block_resident_bytes(wl.d, wl.io_dtype)
+    return int(max(1, min(wl.blocks, (int(free_bytes) - int(reserve_bytes)) // per)))
+
+
 def _gen(device, seed):
     g = torch.Generator(device=device)
     g.manual_seed(seed)

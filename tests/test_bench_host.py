@@ -82,3 +82,43 @@ def test_reference_arm_runs_on_rank_zero_only():
     assert line["impl"] == "reference" and line["unit"] == "ms/step" and line["higher_is_better"] is False
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["value"] > 0
+
+
+def test_gpus_flag_launches_the_ranks_and_partitions_whole_matrices():
+    """`bench.py --gpus 2` with no launcher around it starts two ranks itself
+    (gloo on CPU in --dry-run).  Under --partition matrices every matrix of the
+    set belongs to exactly one rank, and the printed line says n_gpus: 2."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR",
+                                                            "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--partition", "matrices",
+                        "--config", "2", "--dry-run"], env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-800:]
+    lines = [json.loads(x) for x in r.stdout.splitlines() if x.startswith("{")]
+    assert len(lines) == 1, "rank 0 alone prints"
+    line = lines[0]
+    assert line["n_gpus"] == 2 and line["scaling"] == "strong" and line["partition"] == "matrices"
+    lists = line["matrix_lists"]
+    n = len(workload(2).shapes)
+    assert len(lists) == 2
+    assert sorted(lists[0] + lists[1]) == list(range(n)), "union is the whole set, no matrix twice"
+    assert not set(lists[0]) & set(lists[1])
+    cost = line["ns5_flop_per_rank"]
+    assert max(cost) <= 1.1 * (sum(cost) / 2), "balanced within 10 % of the mean"
+    # the same lists as the host planner gives directly
+    owner, _ = B.prm_partition_matrices([tuple(s) for s in workload(2).shapes], 2)
+    assert lists == [[i for i, q in enumerate(owner) if q == k] for k in range(2)]
+
+
+def test_replicas_dry_run_and_world_size_mismatch():
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--config", "2", "--dry-run"],
+                       env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-800:]
+    line = [json.loads(x) for x in r.stdout.splitlines() if x.startswith("{")][0]
+    assert line["n_gpus"] == 2 and line["scaling"] == "weak"
+    assert line["matrix_lists"][0] == line["matrix_lists"][1] == list(range(len(workload(2).shapes)))
+    # a launcher that started another number of ranks than --gpus says is an error, not a silent n_gpus: 1
+    env2 = dict(env, RANK="0", WORLD_SIZE="1", LOCAL_RANK="0")
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--dry-run"], env=env2,
+                       capture_output=True, text=True, timeout=120)
+    assert r.returncode != 0 and "does not match" in r.stderr

@@ -22,10 +22,11 @@ SHAPES = [(256, 512), (256, 1024), (24, 40), (40, 24), (300, 520), (512, 256), (
 @pytest.mark.parametrize("io", ["fp32", "bf16"])
 def test_refresh_tc_direction(shape, io):
     (err,) = _direction_case([shape], io, False, seed=sum(shape))
-    # A 5x5 matrix has too few entries for bf16 rounding to average out: the
-    # same arithmetic that gives ~1e-2 on real shapes scatters between 1e-2
-    # and 3e-2 there, so the tiny case gets twice the bound.
-    assert err <= (TOL if min(shape) >= 16 else 2 * TOL), err
+    assert err <= TOL, err
+    if min(shape) < 64:
+        # fewer than 64 oriented rows: the library refreshes in fp32 (bf16 scatters past
+        # the bound there, tests/test_bf16_emulation.py), so the result is far inside it
+        assert err <= (1e-4 if io == "fp32" else 3e-3), err      # bf16 parameters: the store rounds to 2^-9
 
 
 def test_refresh_tc_groups_and_sub_batches():
@@ -37,18 +38,9 @@ def test_refresh_tc_groups_and_sub_batches():
 
 
 def _structured_case(kind, shapes, check_mode):
-    g = torch.Generator().manual_seed(5)
     cfg = U.oracle_cfg(K=1, nesterov=True, lr=1.0, wd=0.0, scale_mode=0)
     W = [torch.zeros(s, dtype=torch.bfloat16) for s in shapes]
-    G = []
-    for (m, n) in shapes:
-        if kind == "heavy_rows":          # log-normal row scales, as in the 15B-class configuration
-            x = torch.randn(m, n, generator=g) * torch.exp(torch.randn(m, 1, generator=g))
-        elif kind == "low_rank_mild":     # rank-8 signal at the level of the noise
-            x = torch.randn(m, 8, generator=g) @ torch.randn(8, n, generator=g) / 8 ** 0.5 + torch.randn(m, n, generator=g)
-        else:                             # rank-8 spike two orders of magnitude above the noise floor
-            x = torch.randn(m, 8, generator=g) @ torch.randn(8, n, generator=g) + 0.1 * torch.randn(m, n, generator=g)
-        G.append((x * 1e-3).to(torch.bfloat16))
+    G = U.structured_grads(kind, shapes)
     M = [torch.zeros(s) for s in shapes]
     Wg, _ = U.gpu_step(shapes, W, G, M, 0, cfg, "bf16", check_mode)
     errs = []
@@ -64,16 +56,29 @@ def test_refresh_tc_structured_inputs(kind):
     assert max(errs) <= TOL, errs
 
 
+def spiked_bounds(shapes):
+    """1.5 x the error that bf16 storage with fp32 accumulation gives on the
+    very same bits, emulated on the CPU in the order of evaluation the library
+    picks for each shape."""
+    from tests import bf16_emulation as E
+    from tests.test_bf16_emulation import direction_input_of
+    return [1.5 * E.emulated_error(direction_input_of(g, s), E.library_schedule(s))
+            for s, g in zip(shapes, U.structured_grads("spiked", shapes))]
+
+
 def test_refresh_tc_spiked_spectrum_is_bf16_limited():
     # With a few singular values far above the rest, the bf16 rounding of the
     # dominant part is of the order of the small singular values, and NS5
     # amplifies those by ~3.4x per iteration.  That is a property of bf16
-    # operands, not of the kernels: the result stays within 10 % here, and the
-    # fp32 check mode (params stored as bf16 here) is two orders better.
+    # operands, not of the kernels: the CPU emulation of the format gives
+    # 5-6e-2 on this input (tests/test_bf16_emulation.py).  The kernel must
+    # stay within 1.5 x the emulated error; the fp32 check mode (parameters
+    # stored as bf16 here) is two orders better.
     shapes = [(512, 1024)]
     fast = _structured_case("spiked", shapes, False)
     check = _structured_case("spiked", shapes, True)
-    assert max(fast) <= 0.1, fast
+    for e, bound in zip(fast, spiked_bounds(shapes)):
+        assert e <= bound, (fast, bound)
     assert max(check) <= 3e-3, check
 
 
@@ -105,3 +110,39 @@ def test_refresh_tc_zero_matrix():
     M[0].zero_()
     Wg, Mg = U.gpu_step(shapes, W, G, M, 0, cfg, "fp32", False)
     np.testing.assert_allclose(Wg[0], (1 - 5e-5) * U.to_np64(W[0]), rtol=1e-6)
+
+
+def test_refresh_follows_parameters_that_move_on_a_live_handle():
+    """The staged final update reaches the parameters through tensor maps kept
+    in the workspace.  When the caller hands the same handle other parameter
+    buffers, the maps are rewritten; the next refresh must use the new ones
+    (and leave the old buffers alone), wide and tall."""
+    shapes = [(256, 512), (512, 256), (1024, 2560)]
+    cfg = U.oracle_cfg(K=1, nesterov=True, lr=5e-3, wd=0.01)
+    W, G, M = U.make_inputs(shapes, 31, "bf16", grad_std=1e-3, mom_std=1e-3)
+    opt = B.PeriodicRowwiseMuon(shapes, cfg.K, cfg.beta, cfg.nesterov, cfg.lr, cfg.wd)
+    A = [U.Guarded(w) for w in W]
+    Bm = [U.Guarded(w) for w in W]
+    g = [x.cuda() for x in G]
+    mA = [x.cuda() for x in M]
+    mB = [x.cuda() for x in M]
+    opt.step([x.t for x in A], g, mA, 0)
+    torch.cuda.synchronize()
+    A_after = [x.t.clone() for x in A]
+    opt.step([x.t for x in Bm], g, mB, 0)          # same handle, parameters elsewhere; A stays allocated
+    torch.cuda.synchronize()
+    assert opt.status() == B.PRM_OK
+    for i, s in enumerate(shapes):
+        assert A[i].intact() and Bm[i].intact()
+        assert torch.equal(A[i].t, A_after[i]), f"{s}: the old parameter buffer was written again"
+        assert torch.equal(Bm[i].t, A_after[i]), f"{s}: same inputs, same handle, other buffer: same bits"
+        Wr, _ = O.step_matrix(U.to_np64(W[i]), U.to_np64(G[i]), U.to_np64(M[i]), 0, cfg)
+        w0 = U.to_np64(W[i])
+        d_gpu = (1 - cfg.lr * cfg.wd) * w0 - U.to_np64(Bm[i].t)
+        d_ref = (1 - cfg.lr * cfg.wd) * w0 - Wr
+        # The update (~5e-3 * 1/sqrt(c) per element) is small against the half ulp of bf16
+        # parameters of size ~2e-2, so the direction read back through them is coarse: the
+        # parameters must agree closely, the recovered direction roughly.
+        assert np.abs(U.to_np64(Bm[i].t) - Wr).max() <= 1e-3, s
+        assert U.rel_fro(d_gpu, d_ref) <= 0.5, s
+    opt.close()

@@ -48,6 +48,28 @@ def make_inputs(shapes, seed, io, grad_std=1.0, mom_std=0.1, heavy=False):
     return W, G, M
 
 
+def structured_grads(kind, shapes, seed=5, scale=1e-3):
+    """Seeded bf16 gradient matrices with a chosen spectrum: "heavy_rows"
+    (log-normal row scales, as in the 15B-class configuration),
+    "low_rank_mild" (rank-8 signal at the level of the noise), "spiked" (rank-8
+    signal two orders of magnitude above the noise floor), "gauss"."""
+    g = torch.Generator().manual_seed(seed)
+    out = []
+    for (m, n) in shapes:
+        if kind == "heavy_rows":
+            x = torch.randn(m, n, generator=g) * torch.exp(torch.randn(m, 1, generator=g))
+        elif kind == "low_rank_mild":
+            x = torch.randn(m, 8, generator=g) @ torch.randn(8, n, generator=g) / 8 ** 0.5 + torch.randn(m, n, generator=g)
+        elif kind == "spiked":
+            x = torch.randn(m, 8, generator=g) @ torch.randn(8, n, generator=g) + 0.1 * torch.randn(m, n, generator=g)
+        elif kind == "gauss":
+            x = torch.randn(m, n, generator=g)
+        else:
+            raise ValueError(kind)
+        out.append((x * scale).to(torch.bfloat16))
+    return out
+
+
 def oracle_cfg(**kw):
     return O.OracleConfig(**kw)
 

@@ -518,12 +518,8 @@ def main(argv=None):
                                 ns_workspace_bytes=ns_cap, device=dev)
     gram_iters = {(g["rows"], g["cols"]): g["gram_iters"] for g in opt.groups()}
     exec_flop = {(g["rows"], g["cols"]): g["ns5_flop"] for g in opt.groups()}
-    params, moms = [], []
-    for i in range(n):
-        params.append(make_param(wl, i, dev))
-        moms.append(make_momentum(wl, i, dev))
-        if i % 5 == 4:
-            torch.cuda.empty_cache()             # the generators' fp32 temporaries
+    params = [make_param(wl, i, dev) for i in range(n)]
+    moms = [make_momentum(wl, i, dev) for i in range(n)]
     # Gradients: every matrix owns its gradient buffer in HBM.  Two full sets (seeded for step 0 and
     # step 1) alternate from step to step where a second set fits beside the shape set; otherwise
     # one set is reused (timing does not depend on the values).
@@ -532,12 +528,7 @@ def main(argv=None):
     n_sets = 2 if free_now - 2 * grad_bytes > RESERVE_BYTES else 1
     grad_sets = []
     for sset in range(n_sets):
-        gs = []
-        for i in range(n):
-            gs.append(make_grad(wl, i, sset, dev))
-            if i % 5 == 4:
-                torch.cuda.empty_cache()
-        grad_sets.append(gs)
+        grad_sets.append([make_grad(wl, i, sset, dev) for i in range(n)])
     grads = grad_sets[0]
     torch.cuda.synchronize()
 
@@ -624,6 +615,7 @@ def main(argv=None):
     # (PRM_OPT_NS_GRAM_SPAN = 0), on the same buffers, so that the line carries both figures.
     printed = None
     if any(gram_iters.values()) and not args.check_mode and not args.no_printed:
+        torch.cuda.empty_cache()
         opt0 = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
                                      io_dtype=wl.io_dtype, gram_span=0, ns_workspace_bytes=ns_cap, device=dev)
         p0 = [torch.cuda.Event(enable_timing=True) for _ in range(4)]

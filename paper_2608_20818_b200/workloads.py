@@ -103,6 +103,15 @@ def _gen(device, seed):
     return g
 
 
+def _release_temporaries(device):
+    """Hand the generators' fp32 temporaries back to the driver at once.  Left in
+    torch's cache, such a block is later split by a smaller persistent tensor and
+    can then never be released: on a shape set that nearly fills the device that
+    fragmentation costs several GiB."""
+    if torch.device(device).type == "cuda":
+        torch.cuda.empty_cache()
+
+
 def make_param(wl: Workload, idx: int, device="cpu"):
     """Initial parameter W ~ N(0, 0.02^2), rounded to bf16.  In fp32-I/O
     workloads the bf16 values are widened back to fp32 so the same data can
@@ -110,8 +119,12 @@ def make_param(wl: Workload, idx: int, device="cpu"):
     m, n = wl.shapes[idx]
     g = _gen(device, SEED_BASE + 100 * wl.config_id + 7919 * idx + 1)
     w = torch.empty(m, n, dtype=torch.float32, device=device).normal_(0.0, 0.02, generator=g)
-    w = w.to(torch.bfloat16)
-    return w.float() if wl.io_dtype == "fp32" else w
+    out = w.to(torch.bfloat16)
+    if wl.io_dtype == "fp32":
+        out = out.float()
+    del w
+    _release_temporaries(device)
+    return out
 
 
 def make_grad(wl: Workload, idx: int, step: int, device="cpu"):
@@ -122,9 +135,14 @@ def make_grad(wl: Workload, idx: int, step: int, device="cpu"):
     x = torch.empty(m, n, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=g)
     if wl.heavy_tail_rows:
         z = torch.empty(m, 1, dtype=torch.float32, device=device).normal_(0.0, 1.0, generator=g)
-        x = x * torch.exp(z)
-    x = x * wl.grad_std
-    return x if wl.io_dtype == "fp32" else x.to(torch.bfloat16)
+        x.mul_(torch.exp(z))
+    x.mul_(wl.grad_std)
+    if wl.io_dtype == "fp32":
+        return x
+    out = x.to(torch.bfloat16)
+    del x
+    _release_temporaries(device)
+    return out
 
 
 def make_momentum(wl: Workload, idx: int, device="cpu"):

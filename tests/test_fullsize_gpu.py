@@ -68,13 +68,9 @@ def _run_config(config_id, blocks, oracle_shapes, ns_workspace_bytes=None):
     n = len(wl.shapes)
     dev = "cuda"
     rng = np.random.default_rng(config_id)
-    params, moms, grads = [], [], []
-    for i in range(n):
-        params.append(make_param(wl, i, dev))
-        moms.append(make_momentum(wl, i, dev))
-        grads.append(make_grad(wl, i, 0, dev))
-        if i % 5 == 4:
-            torch.cuda.empty_cache()          # the generators' fp32 temporaries
+    params = [make_param(wl, i, dev) for i in range(n)]
+    moms = [make_momentum(wl, i, dev) for i in range(n)]
+    grads = [make_grad(wl, i, 0, dev) for i in range(n)]
     opt = B.PeriodicRowwiseMuon(wl.shapes, wl.K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
                                 ns_workspace_bytes=ns_workspace_bytes)
     block = int(rng.integers(0, n // 5))

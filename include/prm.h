@@ -88,7 +88,16 @@ extern "C" {
  * The check mode always runs the iterations as printed.  Before set_workspace
  * (the workspace holds two more r x r matrices per refreshed matrix with 1 or 2). */
 #define PRM_OPT_NS_GRAM_SPAN 12
-
+/* Which kernels take the row step (rho_t = 0) of TALL matrices, where RowNorm
+ * (Eq. rownorm, on the transposed matrix of Section 3.1) normalises stored columns:
+ *   0 (default), 1: two passes over gradient and momentum (20 bytes per element);
+ *   2: one pass over HBM (14 bytes per element: the data waits in shared memory
+ *      for the column norms) for bf16 matrices with cols % 8 == 0 and at most
+ *      ~25000 rows, two passes for the rest.  Fewer bytes, but bound by the SMs'
+ *      instruction issue: faster than the two passes at full SM clock, slower at
+ *      the reduced clock that follows a power-capped refresh.
+ * Both give the same result up to the order of the fp32 sums.  Before set_workspace. */
+#define PRM_OPT_TALL_KERNEL 13
 
 
 typedef struct prm_ctx prm_ctx;

@@ -26,16 +26,18 @@ struct prm_ctx {
   float gamma_ns = 1.f;   // multiplier on the NS5 branch (ablation: "scalar-controlled" uses gamma)
   int no_refresh = 0;     // ablation: RowNorm at every step
   int gram_span = 2;      // NS5 schedule of the tensor-core path (PRM_OPT_NS_GRAM_SPAN)
+  int tall_kernel = 0;    // row step of tall groups (PRM_OPT_TALL_KERNEL): 0 auto, 1 two passes, 2 streaming where possible
 
   std::vector<Group> groups;
   std::vector<int> group_of_mat, order_in_group, slot_of_mat;   // slot = index in pointer tables
 
   // workspace layout (byte offsets)
-  size_t off_status = 0, off_tables = 0, off_pmaps = 0, off_fro = 0, off_alpha = 0, off_ns = 0, total_bytes = 0;
+  size_t off_status = 0, off_tables = 0, off_pmaps = 0, off_rmaps = 0, off_fro = 0, off_alpha = 0, off_ns = 0, total_bytes = 0;
   char* ws = nullptr;
   size_t ws_bytes = 0;
   std::vector<void*> host_tables;   // 3*n_mats, grouped order: params | grads | momentum
   std::vector<unsigned char> host_pmaps;   // n_mats tensor maps of 128 bytes over the parameters (table order)
+  std::vector<unsigned char> host_rmaps;   // streaming row step: 3 maps (gradient, momentum, parameters) per matrix
   bool tables_uploaded = false;
 
   TcContext* tc = nullptr;
@@ -103,13 +105,17 @@ static void compute_layout(prm_ctx* c) {
   c->off_status = off; off += 256;
   c->off_tables = off; off = align_up(off + (size_t)3 * c->n_mats * sizeof(void*), 256);
   c->off_pmaps = off;  off = align_up(off + (size_t)128 * c->n_mats, 256);
+  c->off_rmaps = off;  off = align_up(off + (size_t)384 * c->n_mats, 256);
   size_t fro_max = 0, ns_max = 0;
   int batch_max = 1;
   for (Group& g : c->groups) {
     if (g.tall) {
       const size_t nblk = (size_t)((g.rows + kTallRows - 1) / kTallRows);
-      g.tall_scratch_off = off; off = align_up(off + (size_t)g.count * nblk * g.cols * 4, 256);
+      // column partial sums of the two-pass kernels, or the streaming kernel's ring of per-wave sums
+      g.tall_scratch_off = off;
+      off = align_up(off + std::max((size_t)g.count * nblk * g.cols * 4, tall_stream_partial_bytes()), 256);
       g.tall_nu_off = off;      off = align_up(off + (size_t)g.count * g.cols * 4, 256);
+      g.tall_sync_off = off;    off = align_up(off + tall_stream_sync_ints(g.cols, g.count) * sizeof(int), 256);
     }
     // Gram-space iterations trade 6 r^2 (c - r) flop for six r^3 products: worth it
     // from c = 1.5 r on; below 1024 rows the time is noise and the bf16 rounding of the
@@ -183,6 +189,7 @@ extern "C" int prm_create(prm_ctx** out, const int64_t* shapes, int n_mats, int 
     c->slot_of_mat[i] = c->groups[c->group_of_mat[i]].first + c->order_in_group[i];
   c->host_tables.assign((size_t)3 * n_mats, nullptr);
   c->host_pmaps.assign((size_t)128 * n_mats, 0);
+  c->host_rmaps.assign((size_t)384 * n_mats, 0);
   compute_layout(c);
   *out = c;
   return PRM_OK;
@@ -204,6 +211,10 @@ extern "C" int prm_set_option(prm_ctx* c, int key, double v) {
     case PRM_OPT_NO_REFRESH:
       if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
       c->no_refresh = (int)v; return PRM_OK;
+    case PRM_OPT_TALL_KERNEL:
+      if (attached) return fail(c, PRM_ERR_STATE, "option must be set before prm_set_workspace");
+      if (v != 0 && v != 1 && v != 2) return fail(c, PRM_ERR_ARG, "value must be 0, 1 or 2");
+      c->tall_kernel = (int)v; return PRM_OK;
     case PRM_OPT_IO_DTYPE:
     case PRM_OPT_CHECK_MODE:
     case PRM_OPT_NS_GRAM_SPAN:
@@ -239,10 +250,21 @@ extern "C" int prm_set_workspace(prm_ctx* c, void* dev_ptr, size_t bytes) {
   c->ws = (char*)dev_ptr;
   c->ws_bytes = bytes;
   c->tables_uploaded = false;
-  if (!c->check_mode && !c->tc) {
+  if (!c->tc) {
+    // The tensor-core products need this context; the streaming row step only uses it where it
+    // exists (its tensor maps), so the fp32 check mode works without one.
     std::string err;
     c->tc = tc_create(&err);
-    if (!c->tc) { c->ws = nullptr; return fail(c, PRM_ERR_CUDA, "prm_set_workspace: " + err); }
+    if (!c->tc && !c->check_mode) { c->ws = nullptr; return fail(c, PRM_ERR_CUDA, "prm_set_workspace: " + err); }
+  }
+  for (Group& g : c->groups) {
+    g.stream = TallStreamPlan();
+    // The streaming kernel is opt-in: it moves 14 instead of 20 bytes per element, but it is
+    // bound by instruction issue and loses to the two passes at the reduced SM clock that
+    // follows a power-capped refresh (see rowstep_stream.cu).
+    if (!g.tall || !c->tc || c->tall_kernel != 2) continue;
+    const TallStreamPlan p = tall_stream_plan(g.rows, g.cols, c->io_fp32, tc_sm_count(c->tc));
+    if (p.ok) g.stream = p;
   }
   return PRM_OK;
 }
@@ -572,6 +594,22 @@ static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
       ce = cudaMemcpyAsync(c->ws + c->off_pmaps, c->host_pmaps.data(), (size_t)128 * n, cudaMemcpyHostToDevice, stream);
       if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("parameter tensor maps: ") + cudaGetErrorString(ce));
     }
+    bool any_stream = false;
+    for (int i = 0; i < n; ++i) {
+      const Group& g = c->groups[c->group_of_mat[i]];
+      if (!g.stream.ok) continue;
+      any_stream = true;
+      unsigned char* dst = c->host_rmaps.data() + (size_t)384 * c->slot_of_mat[i];
+      const int pw = tall_stream_panel();
+      if (!tc_encode_tile_map(c->tc, grads_dev[i], g.rows, g.cols, 2, pw, g.stream.R, dst) ||
+          !tc_encode_tile_map(c->tc, momentum[i], g.rows, g.cols, 4, pw, g.stream.R, dst + 128) ||
+          !tc_encode_tile_map(c->tc, params[i], g.rows, g.cols, 2, pw, g.stream.R, dst + 256))
+        return fail(c, PRM_ERR_CUDA, "cannot encode the tensor maps of the streaming row step");
+    }
+    if (any_stream) {
+      ce = cudaMemcpyAsync(c->ws + c->off_rmaps, c->host_rmaps.data(), (size_t)384 * n, cudaMemcpyHostToDevice, stream);
+      if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("row-step tensor maps: ") + cudaGetErrorString(ce));
+    }
     c->tables_uploaded = true;
   }
   if (grads_host) {
@@ -622,8 +660,14 @@ static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
       if (rc != PRM_OK) return rc;
     } else {
       ProfScope ps(c, g.tall ? PRM_PROF_ROW_TALL : PRM_PROF_ROW_WIDE, stream);
-      ce = launch_rowstep(t, g, s, c->io_fp32, (float*)(c->ws + g.tall_scratch_off),
-                          (float*)(c->ws + g.tall_nu_off), stream, &c->launches);
+      if (g.tall && g.stream.ok)
+        ce = launch_rowstep_tall_stream(t, g, s, g.stream, c->ws + c->off_rmaps + (size_t)384 * g.first,
+                                        (float*)(c->ws + g.tall_scratch_off), (float*)(c->ws + g.tall_nu_off),
+                                        (int*)(c->ws + g.tall_sync_off), (int*)(c->ws + c->off_status),
+                                        tc_sm_count(c->tc), stream, &c->launches);
+      else
+        ce = launch_rowstep(t, g, s, c->io_fp32, (float*)(c->ws + g.tall_scratch_off),
+                            (float*)(c->ws + g.tall_nu_off), stream, &c->launches);
       if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("row step: ") + cudaGetErrorString(ce));
     }
   }

@@ -41,6 +41,38 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+// The same test, but the hardware may suspend the warp for up to `hint_ns` while
+// the phase is incomplete, so that a waiting warp issues next to nothing.
+__device__ __forceinline__ bool mbar_try_wait_suspend(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait for roles that wait long and often (the streaming row step): the warp sleeps in
+// the barrier instead of polling it.  Same contract as mbar_wait.
+__device__ __forceinline__ bool mbar_wait_quiet(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                int* status, uint64_t limit_ns = kWaitLimitNs) {
+  if (mbar_try_wait(bar, parity)) return true;
+  uint64_t t0 = 0;
+  for (;;) {
+    if (mbar_try_wait_suspend(bar, parity, 20000u)) return true;      // up to 20 us asleep
+    if (*abort_flag) return false;
+    const uint64_t now = global_ns();
+    if (t0 == 0) {
+      t0 = now;
+    } else if (now - t0 > limit_ns) {
+      *abort_flag = 1;
+      atomicOr(status, kStatusTimeout);
+      return false;
+    }
+  }
+}
 // Bounded wait.  Returns false if the CTA is aborting (this or another role
 // ran out of time); the first to give up raises the device status word.
 // The global timer and the abort flag are looked at only every 64th poll, which

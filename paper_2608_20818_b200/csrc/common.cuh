@@ -156,6 +156,16 @@ struct PtrTables {
   float** momentum;       // [n_mats]
 };
 
+// Launch geometry of the streaming (single-pass) row step of a tall group; ok = 0
+// where the group does not qualify and the two-pass kernels run instead.
+struct TallStreamPlan {
+  int ok = 0;
+  int R = 0;        // rows per CTA slab
+  int lag = 0;      // waves between a slab's two phases
+  int depth = 0;    // waves of tiles the producer keeps in flight
+  size_t smem = 0;  // dynamic shared memory per CTA
+};
+
 struct Group {
   int64_t rows = 0, cols = 0;   // stored shape
   int count = 0;                // matrices in the group
@@ -169,6 +179,9 @@ struct Group {
   int ns_fp32 = 0;              // 1: NS5 of this group runs in fp32 on CUDA cores (check mode, or a tiny matrix)
   size_t tall_scratch_off = 0;  // byte offset of column partials (tall groups)
   size_t tall_nu_off = 0;       // byte offset of column norms (tall groups)
+  size_t tall_sync_off = 0;     // streaming row step: abort flag, per-wave counters and flags
+  size_t tall_maps_off = 0;     // streaming row step: three tensor maps per matrix
+  TallStreamPlan stream;        // filled when the workspace is attached (needs the SM count)
 };
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }

@@ -61,6 +61,21 @@ cudaError_t launch_rowstep(const PtrTables& t, const Group& g, const StepScalars
                            float* tall_partial, float* tall_nu, cudaStream_t stream,
                            int64_t* launches);
 
+// Streaming row step of a tall group (rowstep_stream.cu): one pass over HBM,
+// bf16 parameters and gradients with cols % 8 == 0.  maps_dev: three 128-byte
+// tensor maps per matrix of the group (gradient, momentum, parameters; boxes of
+// plan.R rows x tall_stream_panel() columns, no swizzle) in device memory.
+// partial: tall_stream_partial_bytes(); sync: tall_stream_sync_ints() ints
+// (zeroed by the launcher on the stream).  n_cta CTAs, one per SM, launched
+// cooperatively.
+TallStreamPlan tall_stream_plan(int64_t rows, int64_t cols, int io_fp32, int n_cta);
+size_t tall_stream_partial_bytes();
+size_t tall_stream_sync_ints(int64_t cols, int count);
+int tall_stream_panel();
+cudaError_t launch_rowstep_tall_stream(const PtrTables& t, const Group& g, const StepScalars& s,
+                                       const TallStreamPlan& plan, const void* maps_dev, float* partial, float* nu,
+                                       int* sync, int* status, int n_cta, cudaStream_t stream, int64_t* launches);
+
 // Momentum update + direction input written to the NS5 workspace as the
 // oriented matrix X (r_p x c_p, zero padded), with per-CTA partial sums of
 // squares, then alpha per matrix.  x_fp32: workspace element type (1: fp32
@@ -103,6 +118,11 @@ struct TcContext;
 cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue& ep, int* status,
                            cudaStream_t stream, int64_t* launches);
 bool tc_encode_param_map(TcContext* tc, const void* base, int64_t rows, int64_t cols, int tall, void* out128);
+// Plain (unswizzled) 2-D map over a row-major rows x cols matrix of 2- or 4-byte elements,
+// box = box_rows x box_cols; parts of a box outside the matrix read as zero.
+bool tc_encode_tile_map(TcContext* tc, const void* base, int64_t rows, int64_t cols, int elem_bytes, int box_cols,
+                        int box_rows, void* out128);
+int tc_sm_count(const TcContext* tc);
 TcContext* tc_create(std::string* err);
 // One thread waits limit_ns on a barrier that never completes, then raises
 // the status word (bit kStatusTimeout) and sets *gave_up (device int, may be null).

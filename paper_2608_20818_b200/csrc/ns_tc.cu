@@ -762,6 +762,26 @@ bool tc_encode_param_map(TcContext* tc, const void* base, int64_t rows, int64_t 
   return true;
 }
 
+bool tc_encode_tile_map(TcContext* tc, const void* base, int64_t rows, int64_t cols, int elem_bytes, int box_cols,
+                        int box_rows, void* out128) {
+  if (!tc || (elem_bytes != 2 && elem_bytes != 4) || ((uintptr_t)base & 15) != 0) return false;
+  if ((cols * elem_bytes) % 16 != 0 || box_cols < 1 || box_cols > 256 || box_rows < 1 || box_rows > 256) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * (cuuint64_t)elem_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMap m;
+  CUresult r = tc->encode(&m, elem_bytes == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                          const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return false;
+  memcpy(out128, &m, sizeof(CUtensorMap));
+  return true;
+}
+
+int tc_sm_count(const TcContext* tc) { return tc ? tc->sm_count : 0; }
+
 cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue& ep, int* status,
                            cudaStream_t stream, int64_t* launches) {
   if (!tc) return cudaErrorInvalidValue;

@@ -135,7 +135,9 @@ static void compute_layout(prm_ctx* c) {
     g.ns_batch = nb;
 
     ns_max = std::max(ns_max, per_mat * nb);
-    fro_max = std::max(fro_max, (size_t)nb * (size_t)((g.rp / 64) * (g.cp / 64)));
+    // one partial per CTA of the pre-pass: 64 x 64 tiles (tall), or 4 rows x 2048 columns (wide)
+    fro_max = std::max(fro_max, (size_t)nb * std::max((size_t)((g.rp / 64) * (g.cp / 64)),
+                                                      (size_t)((g.rp / 4) * ((g.cp + 2047) / 2048))));
     batch_max = std::max(batch_max, nb);
   }
   c->off_fro = off;   off = align_up(off + fro_max * 4, 256);

@@ -95,6 +95,67 @@ ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
   }
 }
 
+// Wide matrices need no transposition, so no shared-memory tile: a CTA streams
+// kWideRows rows x kWideCols columns, every thread holding one 8-element vector
+// of each row, all loads issued before the first use (12 outstanding 16-byte
+// loads per thread with bf16 gradients).  Rows and columns of the padded
+// workspace extent that lie outside the matrix are written as zeros.
+constexpr int kWideRows = 4;
+constexpr int kWideCols = kPreThreads * 8;
+
+template <typename IO, typename XT_>
+__global__ void __launch_bounds__(kPreThreads)
+ns_prepass_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
+                       XT_* __restrict__ X, int64_t ld_x, int64_t bs_x, int prow,
+                       float* __restrict__ fro_partial) {
+  __shared__ float warp_part[kPreThreads / 32];
+  const int b = blockIdx.z;
+  const IO* __restrict__ g = reinterpret_cast<const IO*>(t.grads[first + b]);
+  float* __restrict__ m = t.momentum[first + b];
+  XT_* __restrict__ x = X + (int64_t)b * bs_x;
+  const int col = blockIdx.x * kWideCols + threadIdx.x * 8;
+  const int row0 = blockIdx.y * kWideRows;
+  const bool col_in = col < cols;             // cols % 8 == 0: the whole vector is inside or outside
+  float gv[kWideRows][8], mv[kWideRows][8];
+#pragma unroll
+  for (int k = 0; k < kWideRows; ++k) {
+    if (col_in && row0 + k < rows) {
+      const int64_t off = (int64_t)(row0 + k) * cols + col;
+      load8_stream(g + off, gv[k]);
+      load8_stream(m + off, mv[k]);
+    }
+  }
+  float acc = 0.f;
+#pragma unroll
+  for (int k = 0; k < kWideRows; ++k) {
+    const int row = row0 + k;
+    float u[8];
+    if (col_in && row < rows) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const float mn = blend(s.beta, mv[k][e], s.omb, gv[k][e]);
+        mv[k][e] = mn;
+        u[e] = s.nesterov ? blend(s.beta, mn, s.omb, gv[k][e]) : mn;
+        acc += u[e] * u[e];
+      }
+      store8(m + (int64_t)row * cols + col, mv[k]);
+    } else {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) u[e] = 0.f;
+    }
+    if (col < ld_x && row < prow) store8(x + (int64_t)row * ld_x + col, u);
+  }
+  acc = warp_sum(acc);
+  if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < kPreThreads / 32; ++w) tot += warp_part[w];
+    fro_partial[((int64_t)b * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x] = tot;
+  }
+}
+
 // alpha[b] = 1/(sqrt(sum of partials) + eps_ns); one CTA per matrix, fixed
 // summation order.
 __global__ void __launch_bounds__(kPreThreads)
@@ -127,9 +188,18 @@ static cudaError_t prepass_inst(const PtrTables& t, const Group& g, int first, i
   XT_* straight = g.tall ? nullptr : X;
   XT_* transposed = g.tall ? X : nullptr;
   const int64_t bs = g.rp * g.cp;
+  const bool vec = (g.cols % 8 == 0);
+  if (!g.tall && vec) {
+    dim3 gw((unsigned)((pcol + kWideCols - 1) / kWideCols), (unsigned)(prow / kWideRows), (unsigned)batch);
+    if (gw.y <= 65535 && gw.z <= 65535) {
+      ns_prepass_wide_kernel<IO, XT_><<<gw, kPreThreads, 0, stream>>>(t, first, (int)g.rows, (int)g.cols, s, X, pcol, bs,
+                                                                        (int)prow, fro_partial);
+      ns_alpha_kernel<<<batch, kPreThreads, 0, stream>>>(fro_partial, (int)(gw.x * gw.y), s.eps_ns, alpha);
+      return cudaGetLastError();
+    }
+  }
   dim3 grid((unsigned)(pcol / kPreTile), (unsigned)(prow / kPreTile), (unsigned)batch);
   if (grid.y > 65535 || grid.z > 65535) return cudaErrorInvalidValue;
-  const bool vec = (g.cols % 8 == 0);
   if (vec)
     ns_prepass_kernel<IO, XT_, true><<<grid, kPreThreads, 0, stream>>>(
         t, first, (int)g.rows, (int)g.cols, s, straight, pcol, bs, transposed, prow, bs, fro_partial);

@@ -398,6 +398,15 @@ PRM_API int prm_pipeline_model(const double* a, const double* c, int n_buckets, 
 PRM_API int prm_partition_matrices(const int64_t* shapes, int n_mats, int world, int* owner_of_mat,
                                    double* cost_out);
 
+/*
+ * The shape-dependent update scale s(W) of Eq. finite_ns5 for a stored
+ * rows x cols matrix under PRM_OPT_SCALE_MODE `mode` (the paper names s(W) and
+ * does not define it; the modes are listed at the option).  Host only.  A
+ * caller that applies the row step to a row SHARD (prm_tall_shard_apply) passes
+ * the scale of the whole matrix, which this returns; 0 on a bad argument.
+ */
+PRM_API double prm_shape_scale(int mode, int64_t rows, int64_t cols);
+
 /* Frees host resources.  Device memory belongs to the caller. */
 PRM_API int prm_destroy(prm_ctx* ctx);
 

@@ -46,7 +46,7 @@ EXPORTS = (
     "prm_profile", "prm_profile_read", "prm_rowstep_tall_noalloc", "prm_selftest_timeout", "prm_adamw_step",
     "prm_tall_shard_scratch_bytes", "prm_tall_shard_stats", "prm_tall_shard_apply", "prm_group_info",
     "prm_shard_rows", "prm_bucket_plan", "prm_shard_momentum_pack", "prm_refresh_gathered", "prm_refresh_segments", "prm_pipeline_model",
-    "prm_partition_matrices",
+    "prm_partition_matrices", "prm_shape_scale",
 )
 PRM_PROF_ROW_WIDE, PRM_PROF_ROW_TALL, PRM_PROF_PREPASS, PRM_PROF_GRAM = 0, 1, 2, 3
 PRM_PROF_POLY, PRM_PROF_UPDATE, PRM_PROF_UPDATE_FINAL, PRM_PROF_GRAMSPACE, PRM_PROF_COUNT = 4, 5, 6, 7, 8
@@ -137,6 +137,8 @@ def lib():
     L.prm_pipeline_model.restype = c_int
     L.prm_partition_matrices.argtypes = [POINTER(c_int64), c_int, c_int, POINTER(c_int), POINTER(c_double)]
     L.prm_partition_matrices.restype = c_int
+    L.prm_shape_scale.argtypes = [c_int, c_int64, c_int64]
+    L.prm_shape_scale.restype = c_double
     _lib_handle = L
     return L
 
@@ -364,6 +366,14 @@ def prm_partition_matrices(shapes, world):
     if code != PRM_OK:
         raise PrmError(code, "prm_partition_matrices: bad argument")
     return list(owner)[:n], list(cost)[:int(world)]
+
+
+def prm_shape_scale(mode, rows, cols):
+    """s(W) for a stored rows x cols matrix under PRM_OPT_SCALE_MODE `mode`."""
+    v = float(lib().prm_shape_scale(int(mode), int(rows), int(cols)))
+    if v == 0.0:
+        raise PrmError(PRM_ERR_ARG, "prm_shape_scale: bad argument")
+    return v
 
 
 def prm_destroy(h):

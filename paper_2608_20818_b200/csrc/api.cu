@@ -749,6 +749,11 @@ extern "C" int prm_selftest_timeout(prm_ctx* c, double limit_ms, void* cuda_stre
   return PRM_OK;
 }
 
+extern "C" double prm_shape_scale(int mode, int64_t rows, int64_t cols) {
+  if (mode < 0 || mode > 2 || rows < 1 || cols < 1) return 0.0;
+  return (double)shape_scale(mode, rows, cols);
+}
+
 extern "C" const char* prm_last_error(const prm_ctx* c) { return c ? c->err.c_str() : g_create_err.c_str(); }
 
 extern "C" int64_t prm_launch_count(const prm_ctx* c) { return c ? c->launches : 0; }

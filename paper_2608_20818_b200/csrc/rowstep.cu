@@ -12,12 +12,13 @@
 #include <cooperative_groups.h>
 
 #include "launch.cuh"
+#include "tall_kernels.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace prm {
 
-constexpr int kRowThreads = 256;
+constexpr int kRowThreads = kTallThreads;
 
 // ------------------------------------------------------------------ wide
 // One row per CTA of THREADS threads (or per cluster of CLUSTER CTAs for very
@@ -143,59 +144,43 @@ rowstep_wide_generic_kernel(PtrTables t, int first, int rows, int cols, StepScal
 
 // ------------------------------------------------------------------ tall
 // Pass 1: momentum update and per-column partial sums of squares over a block
-// of kTallRows rows.  A lane owns V consecutive columns; the 8 warps of a CTA
-// take interleaved rows and are combined in a fixed order.
+// of kTallRows rows.  Matrices whose column count is a multiple of 8 run the
+// shared vector bodies (tall_kernels.cuh); the rest a scalar version with one
+// column per lane.
 template <typename IO, int V>
 __global__ void __launch_bounds__(kRowThreads)
 rowstep_tall_pass1_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
                           float* __restrict__ partial /*[count][row blocks][cols]*/) {
-  __shared__ float red[kRowThreads / 32][32 * V + 1];
   const int mat = blockIdx.z;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int col0 = (blockIdx.x * 32 + lane) * V;
   const int row0 = blockIdx.y * kTallRows;
   const int row1 = min(rows, row0 + kTallRows);
   const IO* __restrict__ g = reinterpret_cast<const IO*>(t.grads[first + mat]);
   float* __restrict__ m = t.momentum[first + mat];
-  float cs[V];
-#pragma unroll
-  for (int e = 0; e < V; ++e) cs[e] = 0.f;
-  if (col0 < cols) {
-#pragma unroll 4
-    for (int row = row0 + warp; row < row1; row += kRowThreads / 32) {
-      const int64_t off = (int64_t)row * cols + col0;
-      if constexpr (V == 8) {
-        float gv[8], mv[8];
-        load8_stream(g + off, gv);
-        load8(m + off, mv);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float mn = blend(s.beta, mv[e], s.omb, gv[e]);
-          mv[e] = mn;
-          const float uu = s.nesterov ? blend(s.beta, mn, s.omb, gv[e]) : mn;
-          cs[e] += uu * uu;
-        }
-        store8(m + off, mv);
-      } else {
+  float* prow = partial + ((int64_t)mat * gridDim.y + blockIdx.y) * cols;
+  if constexpr (V == 8) {
+    tall_pass1_block<IO>(g, m, cols, row0, row1, blockIdx.x, s.beta, s.omb, s.nesterov, prow);
+  } else {
+    __shared__ float red[kRowThreads / 32][33];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int col = blockIdx.x * 32 + lane;
+    float cs = 0.f;
+    if (col < cols) {
+      for (int row = row0 + warp; row < row1; row += kRowThreads / 32) {
+        const int64_t off = (int64_t)row * cols + col;
         const float gv = to_f32(g[off]);
         const float mn = blend(s.beta, m[off], s.omb, gv);
         m[off] = mn;
         const float uu = s.nesterov ? blend(s.beta, mn, s.omb, gv) : mn;
-        cs[0] += uu * uu;
+        cs += uu * uu;
       }
     }
-  }
-#pragma unroll
-  for (int e = 0; e < V; ++e) red[warp][lane * V + e] = cs[e];
-  __syncthreads();
-  const int nblk = gridDim.y;
-  for (int cl = threadIdx.x; cl < 32 * V; cl += kRowThreads) {
-    const int col = blockIdx.x * 32 * V + cl;
-    if (col < cols) {
+    red[warp][lane] = cs;
+    __syncthreads();
+    if (threadIdx.x < 32 && col < cols) {
       float tot = 0.f;
 #pragma unroll
-      for (int w = 0; w < kRowThreads / 32; ++w) tot += red[w][cl];
-      partial[((int64_t)mat * nblk + blockIdx.y) * cols + col] = tot;
+      for (int w = 0; w < kRowThreads / 32; ++w) tot += red[w][threadIdx.x];
+      prow[col] = tot;
     }
   }
 }
@@ -207,10 +192,7 @@ rowstep_tall_colnorm_kernel(const float* __restrict__ partial, float* __restrict
   const int mat = blockIdx.y;
   const int col = blockIdx.x * kRowThreads + threadIdx.x;
   if (col >= cols) return;
-  const float* src = partial + (int64_t)mat * nblk * cols + col;
-  float tot = 0.f;
-  for (int b = 0; b < nblk; ++b) tot += src[(int64_t)b * cols];
-  nu[(int64_t)mat * cols + col] = fmaxf(sqrtf(tot), eps);
+  nu[(int64_t)mat * cols + col] = fmaxf(sqrtf(tall_column_sum(partial + (int64_t)mat * nblk * cols, nblk, cols, col)), eps);
 }
 
 // Pass 2: scale by the column norms and update the parameters.
@@ -219,37 +201,26 @@ __global__ void __launch_bounds__(kRowThreads)
 rowstep_tall_pass2_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
                           const float* __restrict__ nu /*[count][cols]*/) {
   const int mat = blockIdx.z;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int col0 = (blockIdx.x * 32 + lane) * V;
-  if (col0 >= cols) return;
   const int row0 = blockIdx.y * kTallRows;
   const int row1 = min(rows, row0 + kTallRows);
   const IO* __restrict__ g = reinterpret_cast<const IO*>(t.grads[first + mat]);
   const float* __restrict__ m = t.momentum[first + mat];
   IO* __restrict__ p = reinterpret_cast<IO*>(t.params[first + mat]);
-  float coef[V];
-#pragma unroll
-  for (int e = 0; e < V; ++e) coef[e] = s.lr_s * s.gamma / nu[(int64_t)mat * cols + col0 + e];
-#pragma unroll 4
-  for (int row = row0 + warp; row < row1; row += kRowThreads / 32) {
-    const int64_t off = (int64_t)row * cols + col0;
-    if constexpr (V == 8) {
-      float mv[8], pv[8];
-      load8_stream(m + off, mv);
-      load8_stream(p + off, pv);
-      if (s.nesterov) {
-        float gv[8];
-        load8_stream(g + off, gv);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) mv[e] = blend(s.beta, mv[e], s.omb, gv[e]);
-      }
-#pragma unroll
-      for (int e = 0; e < 8; ++e) pv[e] = s.decay * pv[e] - coef[e] * mv[e];
-      store8(p + off, pv);
-    } else {
+  const float* nu_m = nu + (int64_t)mat * cols;
+  const float k = s.lr_s * s.gamma;
+  if constexpr (V == 8) {
+    tall_pass2_block<IO>(p, g, m, cols, row0, row1, blockIdx.x, s.beta, s.omb, s.nesterov, s.decay,
+                         [&](int col) { return k / nu_m[col]; });
+  } else {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int col = blockIdx.x * 32 + lane;
+    if (col >= cols) return;
+    const float coef = k / nu_m[col];
+    for (int row = row0 + warp; row < row1; row += kRowThreads / 32) {
+      const int64_t off = (int64_t)row * cols + col;
       float uu = m[off];
       if (s.nesterov) uu = blend(s.beta, uu, s.omb, to_f32(g[off]));
-      from_f32(p + off, s.decay * to_f32(p[off]) - coef[0] * uu);
+      from_f32(p + off, s.decay * to_f32(p[off]) - coef * uu);
     }
   }
 }

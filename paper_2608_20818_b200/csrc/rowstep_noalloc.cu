@@ -18,14 +18,13 @@
 
 #include <stdio.h>
 
-#include "common.cuh"
+#include "tall_kernels.cuh"
 
 namespace {
 
 using namespace prm;
 
 constexpr size_t kNoAllocFloats = (size_t)1 << 20;
-constexpr int kNaThreads = 256;
 constexpr int kNaMaxDevices = 64;
 
 // In host code this name is only a handle for cudaGetSymbolAddress: it is not
@@ -36,85 +35,30 @@ std::mutex g_na_mutex;
 float* g_na_addr[kNaMaxDevices] = {};   // device address of the array, per device
 
 template <typename IO>
-__global__ void __launch_bounds__(kNaThreads)
+__global__ void __launch_bounds__(kTallThreads)
 na_pass1_kernel(const IO* __restrict__ g, float* __restrict__ m, int rows, int cols, float beta,
                 float omb, int nesterov, float* __restrict__ partial /*[row blocks][cols]*/) {
-  __shared__ float red[kNaThreads / 32][32 * 8 + 1];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int col0 = (blockIdx.x * 32 + lane) * 8;
   const int row0 = blockIdx.y * kTallRows;
-  const int row1 = min(rows, row0 + kTallRows);
-  float cs[8];
-#pragma unroll
-  for (int e = 0; e < 8; ++e) cs[e] = 0.f;
-  if (col0 < cols) {
-#pragma unroll 4
-    for (int row = row0 + warp; row < row1; row += kNaThreads / 32) {
-      const int64_t off = (int64_t)row * cols + col0;
-      float gv[8], mv[8];
-      load8_stream(g + off, gv);
-      load8(m + off, mv);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const float mn = blend(beta, mv[e], omb, gv[e]);
-        mv[e] = mn;
-        const float uu = nesterov ? blend(beta, mn, omb, gv[e]) : mn;
-        cs[e] += uu * uu;
-      }
-      store8(m + off, mv);
-    }
-  }
-#pragma unroll
-  for (int e = 0; e < 8; ++e) red[warp][lane * 8 + e] = cs[e];
-  __syncthreads();
-  const int col = blockIdx.x * 256 + threadIdx.x;
-  if (col < cols) {
-    float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < kNaThreads / 32; ++w) tot += red[w][threadIdx.x];
-    partial[(int64_t)blockIdx.y * cols + col] = tot;
-  }
+  tall_pass1_block<IO>(g, m, cols, row0, min(rows, row0 + kTallRows), blockIdx.x, beta, omb, nesterov,
+                       partial + (int64_t)blockIdx.y * cols);
 }
 
-__global__ void __launch_bounds__(kNaThreads)
+__global__ void __launch_bounds__(kTallThreads)
 na_colnorm_kernel(const float* __restrict__ partial, float* __restrict__ nu, int nblk, int cols,
                   float eps) {
-  const int col = blockIdx.x * kNaThreads + threadIdx.x;
+  const int col = blockIdx.x * kTallThreads + threadIdx.x;
   if (col >= cols) return;
-  float tot = 0.f;
-  for (int b = 0; b < nblk; ++b) tot += partial[(int64_t)b * cols + col];
-  nu[col] = fmaxf(sqrtf(tot), eps);
+  nu[col] = fmaxf(sqrtf(tall_column_sum(partial, nblk, cols, col)), eps);
 }
 
 template <typename IO>
-__global__ void __launch_bounds__(kNaThreads)
+__global__ void __launch_bounds__(kTallThreads)
 na_pass2_kernel(IO* __restrict__ p, const IO* __restrict__ g, const float* __restrict__ m, int rows,
                 int cols, float beta, float omb, int nesterov, float decay, float lr_s_gamma,
                 const float* __restrict__ nu) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int col0 = (blockIdx.x * 32 + lane) * 8;
-  if (col0 >= cols) return;
   const int row0 = blockIdx.y * kTallRows;
-  const int row1 = min(rows, row0 + kTallRows);
-  float coef[8];
-#pragma unroll
-  for (int e = 0; e < 8; ++e) coef[e] = lr_s_gamma / nu[col0 + e];
-#pragma unroll 4
-  for (int row = row0 + warp; row < row1; row += kNaThreads / 32) {
-    const int64_t off = (int64_t)row * cols + col0;
-    float mv[8], pv[8];
-    load8_stream(m + off, mv);
-    load8_stream(p + off, pv);
-    if (nesterov) {
-      float gv[8];
-      load8_stream(g + off, gv);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) mv[e] = blend(beta, mv[e], omb, gv[e]);
-    }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) pv[e] = decay * pv[e] - coef[e] * mv[e];
-    store8(p + off, pv);
-  }
+  tall_pass2_block<IO>(p, g, m, cols, row0, min(rows, row0 + kTallRows), blockIdx.x, beta, omb, nesterov, decay,
+                       [&](int col) { return lr_s_gamma / nu[col]; });
 }
 
 int na_fail(char* errbuf, size_t len, int code, const char* msg) {
@@ -130,10 +74,10 @@ cudaError_t na_launch(void* param, const void* grad, float* momentum, int rows, 
   float* partial = scratch;
   float* nu = scratch + (size_t)nblk * cols;
   dim3 grid((cols + 255) / 256, nblk, 1);
-  na_pass1_kernel<IO><<<grid, kNaThreads, 0, stream>>>((const IO*)grad, momentum, rows, cols, beta,
+  na_pass1_kernel<IO><<<grid, kTallThreads, 0, stream>>>((const IO*)grad, momentum, rows, cols, beta,
                                                        1.f - beta, nesterov, partial);
-  na_colnorm_kernel<<<(cols + kNaThreads - 1) / kNaThreads, kNaThreads, 0, stream>>>(partial, nu, nblk, cols, eps);
-  na_pass2_kernel<IO><<<grid, kNaThreads, 0, stream>>>((IO*)param, (const IO*)grad, momentum, rows, cols,
+  na_colnorm_kernel<<<(cols + kTallThreads - 1) / kTallThreads, kTallThreads, 0, stream>>>(partial, nu, nblk, cols, eps);
+  na_pass2_kernel<IO><<<grid, kTallThreads, 0, stream>>>((IO*)param, (const IO*)grad, momentum, rows, cols,
                                                        beta, 1.f - beta, nesterov, decay, lr_s_gamma, nu);
   return cudaGetLastError();
 }

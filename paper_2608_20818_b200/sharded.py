@@ -19,8 +19,6 @@ injectable so that ordering, packing and slicing can be exercised on CPU ranks.
 
 from __future__ import annotations
 
-import math
-
 import torch
 
 from . import binding as B
@@ -38,8 +36,9 @@ def pack_offsets(cols_list):
 class CudaTallBackend:
     """Marshals one tall shard to the library's two entry points."""
 
-    def __init__(self, beta, nesterov, lr, wd, gamma, eps_row):
+    def __init__(self, beta, nesterov, lr, wd, gamma, eps_row, scale_mode=1):
         self.hp = dict(beta=beta, nesterov=nesterov, lr=lr, wd=wd, gamma=gamma, eps_row=eps_row)
+        self.scale_mode = int(scale_mode)
         self._scratch = None
 
     def stats(self, grad, mom, out, stream):
@@ -54,9 +53,10 @@ class CudaTallBackend:
         if code != B.PRM_OK:
             raise B.PrmError(code, "prm_tall_shard_stats failed")
 
-    def apply(self, param, grad, mom, colsumsq, scale, stream):
+    def apply(self, param, grad, mom, colsumsq, global_rows, stream):
         rows, cols = param.shape
         hp = self.hp
+        scale = B.prm_shape_scale(self.scale_mode, global_rows, cols)      # s(W) of the whole matrix, not of the shard
         code = B.lib().prm_tall_shard_apply(param.data_ptr(), grad.data_ptr(), mom.data_ptr(), rows, cols,
                                             1 if param.dtype == torch.float32 else 0, hp["beta"],
                                             int(bool(hp["nesterov"])), hp["lr"], hp["wd"], hp["gamma"],
@@ -73,7 +73,8 @@ def sharded_row_step(tall, wide_step, backend, group=None, stream=0, stats_dtype
     wide_step  callable running the row step of the locally complete (wide)
                matrices, or None; it is called while the all-reduce is in flight
     backend    object with stats(grad, mom, out, stream) and
-               apply(param, grad, mom, colsumsq, scale, stream)
+               apply(param, grad, mom, colsumsq, global_rows, stream); the shape
+               scale s(W) is the backend's business (it knows the scale mode)
     group      torch.distributed process group (None: default; not initialised:
                single rank, no exchange)
     stats_dtype  element type of the packed statistics (float32 for the CUDA
@@ -97,7 +98,7 @@ def sharded_row_step(tall, wide_step, backend, group=None, stream=0, stats_dtype
         work.wait()                                                   # line 12
     for (p, g, m, global_rows), o in zip(tall, offs):                 # lines 12-13
         cols = p.shape[1]
-        backend.apply(p, g, m, packed[o:o + cols], math.sqrt(max(1.0, global_rows / cols)), stream)
+        backend.apply(p, g, m, packed[o:o + cols], global_rows, stream)
     return packed
 
 
@@ -161,6 +162,19 @@ class SymmetricSendBuffers:
         self.handles[k].barrier()
 
 
+def slot_sizes(bucket_of_mat, offsets, segments):
+    """Elements reserved for each matrix in its bucket's segment, read off the
+    plan: a slot ends where the next slot of the same bucket starts, the last
+    one at the end of the segment."""
+    sizes = [0] * len(offsets)
+    for l, seg in enumerate(segments):
+        members = sorted((offsets[i], i) for i in range(len(offsets)) if bucket_of_mat[i] == l)
+        for k, (off, i) in enumerate(members):
+            end = members[k + 1][0] if k + 1 < len(members) else seg
+            sizes[i] = end - off
+    return sizes
+
+
 def _all_gather(recv, send, group):
     import torch.distributed as td
     try:
@@ -208,6 +222,7 @@ def bucketed_refresh_step(shapes, param_shards, grad_shards, mom_shards, backend
     bucket_of_mat, offsets, segments = backend.plan(shapes, world, bucket_bytes)
     n_buckets = len(segments)
     members = [[i for i in range(n) if bucket_of_mat[i] == l] for l in range(n_buckets)]
+    reserved = slot_sizes(bucket_of_mat, offsets, segments)
     dev = param_shards[0].device
     seg_max = max(segments)
     if buffers is None:
@@ -220,7 +235,7 @@ def bucketed_refresh_step(shapes, param_shards, grad_shards, mom_shards, backend
     stream = torch.cuda.current_stream(dev).cuda_stream if dev.type == "cuda" else 0
     if exchange == "p2p":
         return _refresh_p2p(shapes, param_shards, grad_shards, mom_shards, backend, group, world, rank, buffers,
-                            trace, dist_on, (bucket_of_mat, offsets, segments), members, stream)
+                            trace, dist_on, (bucket_of_mat, offsets, segments), members, reserved, stream)
     if exchange != "allgather":
         raise ValueError("exchange must be 'allgather' or 'p2p'")
     pending = [None, None]
@@ -229,10 +244,8 @@ def bucketed_refresh_step(shapes, param_shards, grad_shards, mom_shards, backend
         send = buffers["send"][l % 2][:segments[l]]
         recv = buffers["recv"][l % 2][:segments[l] * world]
         for i in members[l]:
-            rows, cols = shapes[i]
-            chunk = -(-rows // world)
-            reserved = -(-(chunk * cols) // 8) * 8
-            backend.pack(grad_shards[i], mom_shards[i], cols, reserved, send[offsets[i]:offsets[i] + reserved], stream)
+            backend.pack(grad_shards[i], mom_shards[i], shapes[i][1], reserved[i],
+                         send[offsets[i]:offsets[i] + reserved[i]], stream)
         if trace is not None:
             trace.append(("gather", l))
         if dist_on:
@@ -258,7 +271,7 @@ def bucketed_refresh_step(shapes, param_shards, grad_shards, mom_shards, backend
 
 
 def _refresh_p2p(shapes, param_shards, grad_shards, mom_shards, backend, group, world, rank, buffers, trace,
-                 dist_on, plan, members, stream):
+                 dist_on, plan, members, reserved, stream):
     """Algorithm 2 lines 1-7 with the all-gather folded into the rebuild: the
     segments stay in the send buffers of their owners."""
     bucket_of_mat, offsets, segments = plan
@@ -277,10 +290,8 @@ def _refresh_p2p(shapes, param_shards, grad_shards, mom_shards, backend, group, 
     for l, seg in enumerate(segments):
         send = buffers["send"][l % 2][:seg]
         for i in members[l]:
-            rows, cols = shapes[i]
-            chunk = -(-rows // world)
-            reserved = -(-(chunk * cols) // 8) * 8
-            backend.pack(grad_shards[i], mom_shards[i], cols, reserved, send[offsets[i]:offsets[i] + reserved], stream)
+            backend.pack(grad_shards[i], mom_shards[i], shapes[i][1], reserved[i],
+                         send[offsets[i]:offsets[i] + reserved[i]], stream)
         if symm is not None:
             symm.barrier(l % 2)          # every rank has packed bucket l and is done reading bucket l-2
             ptrs = symm.ptrs(l % 2)

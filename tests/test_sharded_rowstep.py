@@ -32,7 +32,10 @@ class OracleBackend:
         u = O.direction_input(mt, grad.numpy(), HP["beta"], HP["nesterov"])
         out.copy_(torch.from_numpy((u * u).sum(axis=0)))
 
-    def apply(self, param, grad, mom, colsumsq, scale, stream):
+    scale_mode = 1
+
+    def apply(self, param, grad, mom, colsumsq, global_rows, stream):
+        scale = O.shape_scale(global_rows, param.shape[1], self.scale_mode)
         u = O.direction_input(mom.numpy(), grad.numpy(), HP["beta"], HP["nesterov"])
         nu = np.maximum(np.sqrt(colsumsq.numpy()), HP["eps_row"])
         w = (1 - HP["lr"] * HP["wd"]) * param.numpy() - HP["lr"] * scale * HP["gamma"] * u / nu
@@ -109,7 +112,7 @@ def test_shards_on_one_gpu_match_oracle_and_prm_step(io):
         parts.append(out)
     total = torch.stack(parts).sum(dim=0)                            # stands in for the sum all-reduce
     for lo, hi in zip(cuts[:-1], cuts[1:]):
-        be.apply(Wd[lo:hi], Gd[lo:hi], Md[lo:hi], total, math.sqrt(shape[0] / shape[1]), stream)
+        be.apply(Wd[lo:hi], Gd[lo:hi], Md[lo:hi], total, shape[0], stream)
     torch.cuda.synchronize()
     Wr, Mr = O.step_matrix(U.to_np64(W[0]), U.to_np64(G[0]), U.to_np64(M[0]), 1, cfg)
     U.assert_elementwise(U.to_np64(Md), Mr, False, "momentum")
@@ -121,3 +124,38 @@ def test_shards_on_one_gpu_match_oracle_and_prm_step(io):
     torch.cuda.synchronize()
     U.assert_elementwise(U.to_np64(W2), Wg[0], io == "bf16", "param vs prm_step")
     assert np.array_equal(U.to_np64(M2), Mg[0])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("scale_mode", [0, 2])
+def test_sharded_row_step_and_refresh_follow_the_scale_mode(scale_mode):
+    """Both branches of the sharded execution take s(W) from the same option:
+    the row step through the backend's scale mode, the refresh through the
+    handle's."""
+    from paper_2608_20818_b200 import binding as B
+    shape = (1000, 264)
+    cfg = U.oracle_cfg(K=2, scale_mode=scale_mode, **{k: HP[k] for k in ("beta", "nesterov", "lr", "wd", "gamma", "eps_row")})
+    assert B.prm_shape_scale(scale_mode, *shape) == pytest.approx(O.shape_scale(shape[0], shape[1], scale_mode), rel=1e-7)
+    W, G, M = U.make_inputs([shape], 62, "fp32", grad_std=1e-3, mom_std=1e-3)
+    stream = torch.cuda.current_stream().cuda_stream
+    # row step (t = 1) on one shard that is the whole matrix
+    be = S.CudaTallBackend(scale_mode=scale_mode, **HP)
+    W2, G2, M2 = W[0].cuda(), G[0].cuda(), M[0].cuda()
+    S.sharded_row_step([(W2, G2, M2, shape[0])], None, be, stream=stream)
+    torch.cuda.synchronize()
+    Wr, Mr = O.step_matrix(U.to_np64(W[0]), U.to_np64(G[0]), U.to_np64(M[0]), 1, cfg)
+    U.assert_elementwise(U.to_np64(W2), Wr, False, f"row step, scale mode {scale_mode}")
+    # refresh (t = 0) through the bucketed path with one rank, fp32 check mode
+    opt = B.PeriodicRowwiseMuon([shape], cfg.K, cfg.beta, cfg.nesterov, cfg.lr, cfg.wd, scale_mode=scale_mode,
+                                io_dtype="fp32", check_mode=True)
+    W3, G3, M3 = W[0].cuda(), G[0].cuda(), M[0].cuda()
+    S.bucketed_refresh_step([shape], [W3], [G3], [M3], S.CudaRefreshBackend(opt, cfg.beta, cfg.nesterov))
+    torch.cuda.synchronize()
+    assert opt.status() == B.PRM_OK
+    Wr0, _ = O.step_matrix(U.to_np64(W[0]), U.to_np64(G[0]), U.to_np64(M[0]), 0, cfg)
+    w0 = U.to_np64(W[0])
+    d_gpu = (1 - cfg.lr * cfg.wd) * w0 - U.to_np64(W3)
+    d_ref = (1 - cfg.lr * cfg.wd) * w0 - Wr0
+    # the gathered payload is bf16 (2^-9 per element), NS5 itself runs in fp32 here
+    assert U.rel_fro(d_gpu, d_ref) <= 1e-2, U.rel_fro(d_gpu, d_ref)
+    opt.close()

@@ -679,6 +679,7 @@ def main(argv=None):
                    "first_timed_step_index": t_first + args.warmup},
         "refresh_ms": mean_ref if n_ref else None, "row_step_ms": mean_row if n_row else None,
         "refresh_steps_timed": n_ref, "row_steps_timed": n_row,
+        "per_step_ms": [round(t, 3) for t in per_step],       # rank 0, in order; refresh steps are the large ones
         "gpu_launches": launches,
         "clocks": clocks,
         # device time per kernel class over the whole timed region (CUDA events inside the library)

@@ -135,6 +135,11 @@ PRM_API int prm_set_workspace(prm_ctx* ctx, void* dev_ptr, size_t bytes);
  * The branch depends only on step_idx mod K; steps need not be consecutive.
  * cuda_stream is a cudaStream_t (NULL = default stream).  Calls on one handle
  * must be ordered on one stream, or separated by synchronisation.
+ * The first step on a handle, and any step that is given a pointer it has not
+ * seen at that position before, also uploads the pointer tables (and the tensor
+ * maps over the matrices) with host-to-device copies from pageable host memory:
+ * such a step blocks the host until the bytes are staged and cannot run inside
+ * a stream capture.  Steps with unchanged pointers only launch kernels.
  */
 PRM_API int prm_step(prm_ctx* ctx, void* const* params, const void* const* grads,
              float* const* momentum, int64_t step_idx, void* cuda_stream);
@@ -261,8 +266,8 @@ PRM_API int prm_rowstep_tall_noalloc(void* param, const void* grad, float* momen
 
 /*
  * AdamW for the parameters outside the Muon set (Algorithm 1 line 11: biases,
- * normalisation parameters and everything outside the transformer blocks keep
- * "the same AdamW rule as the baseline"; hyper-parameter table: lr 1e-4,
+ * normalisation parameters and everything outside the transformer blocks are
+ * still updated by the baseline's AdamW; hyper-parameter table: lr 1e-4,
  * betas (0.9, 0.95), eps 1e-8, weight decay 0.01).  Decoupled form with bias
  * correction, step >= 1 is the 1-based step count:
  *   p <- p*(1 - lr*wd);  m <- beta1*m + (1-beta1)*g;  v <- beta2*v + (1-beta2)*g^2
@@ -320,7 +325,9 @@ PRM_API int prm_tall_shard_apply(void* param_shard, const void* grad_shard, cons
  * the exchange and the planning; it contains no communication.
  *
  * prm_shard_rows     the row range of one rank (host).
- * prm_bucket_plan    host.  Walks the matrices in caller order; matrix i
+ * prm_bucket_plan    host.  Walks the matrices shape group by shape group
+ *   (groups in order of first appearance, caller order inside a group, so that
+ *   a bucket holds matrices NS5 can batch); matrix i
  *   reserves ceil8(chunk_i * cols_i) elements in every rank's segment
  *   (offset_in_segment[i], a multiple of 8); a new bucket starts when the
  *   gathered payload world * 2 bytes * segment would exceed bucket_bytes (a
@@ -389,8 +396,10 @@ PRM_API int prm_pipeline_model(const double* a, const double* c, int n_buckets, 
  * 1 lines 4-10), so a rank that owns a matrix (parameter, gradient, momentum)
  * runs prm_step on its own list and nothing is exchanged; Section 3.3's
  * collectives exist only because dim-0 sharding splits each matrix.  Host
- * only: longest-processing-time greedy on the NS5 cost 15 r^2 c + 5 r^3 of
- * each matrix (decreasing cost, ties by index; least-loaded rank, ties by
+ * only: longest-processing-time greedy on the NS5 flop the default schedule
+ * executes for each matrix (PRM_OPT_NS_GRAM_SPAN = 2: 8 r^2 c + 13 r^3 where the
+ * Gram-space iterations apply, else 15 r^2 c + 5 r^3; decreasing cost, ties
+ * by index; least-loaded rank, ties by
  * rank).  owner_of_mat[n_mats] receives the rank of each matrix, cost_out[world]
  * (may be NULL) the flop assigned to each rank.  The paper does not describe
  * this layout; it is offered beside the paper's.

@@ -216,8 +216,8 @@ def step(params, grads, momenta, t, cfg: OracleConfig):
 
 
 def adamw_step(p, g, m, v, t, lr=1e-4, beta1=0.9, beta2=0.95, eps=1e-8, wd=0.01):
-    """One AdamW step for a parameter outside the Muon set (Algorithm 1 line 11:
-    "the same AdamW rule as the baseline"; hyper-parameter table: lr 1e-4,
+    """One AdamW step for a parameter outside the Muon set (Algorithm 1 line 11
+    leaves those to the baseline's AdamW; hyper-parameter table: lr 1e-4,
     betas (0.9, 0.95), eps 1e-8, weight decay 0.01).  The paper does not spell
     the rule out; this is the usual decoupled form with bias correction:
         p <- p*(1 - lr*wd)

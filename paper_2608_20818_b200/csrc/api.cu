@@ -117,15 +117,11 @@ static void compute_layout(prm_ctx* c) {
       g.tall_nu_off = off;      off = align_up(off + (size_t)g.count * g.cols * 4, 256);
       g.tall_sync_off = off;    off = align_up(off + tall_stream_sync_ints(g.cols, g.count) * sizeof(int), 256);
     }
-    // Gram-space iterations trade 6 r^2 (c - r) flop for six r^3 products: worth it
-    // from c = 1.5 r on; below 1024 rows the time is noise and the bf16 rounding of the
-    // small r x r matrices averages less well, so those stay on the printed recurrence.
     g.ns_fp32 = (c->check_mode || g.r < kTinyRows) ? 1 : 0;
     const size_t e = g.ns_fp32 ? 4 : 2;
-    g.gram_iters = (!g.ns_fp32 && c->gram_span && g.rp >= 1024 && 2 * g.cp >= 3 * g.rp) ? kGramIters : 0;
-    // Mode 2: beyond c = 2r the Gram matrix of the last iteration is also cheaper from the one
-    // before it (A_4 = P_3 A_3 P_3, two r^3 products) than from X_4 (one r^2 c product).
-    g.last_gram_rec = (g.gram_iters && c->gram_span >= 2 && g.cp > 2 * g.rp) ? 1 : 0;
+    const Ns5Schedule sched = ns5_schedule(g.r, g.c, c->gram_span, g.ns_fp32 != 0);
+    g.gram_iters = sched.gram_iters;
+    g.last_gram_rec = sched.last_gram_rec;
     // X ping-pong, A, B (+ two more r x r matrices for the Gram-space iterations)
     const size_t per_mat = e * (size_t)(2 * g.rp * g.cp + (g.gram_iters ? 4 : 2) * g.rp * g.rp);
     int nb = (int)std::min<size_t>((size_t)g.count, std::max<size_t>(1, c->ns_cap / per_mat));
@@ -290,14 +286,7 @@ extern "C" int prm_group_info(const prm_ctx* c, int group, int64_t* rows, int64_
   if (count) *count = g.count;
   if (ns_batch) *ns_batch = g.ns_batch;
   if (gram_iters) *gram_iters = g.gram_iters;
-  if (ns5_flop) {
-    // X X^T products (r^2 c each, lower blocks), r x c products (2 r^2 c), symmetric r x r products (r^3)
-    const double r = (double)g.r, cc = (double)g.c;
-    const double n_gram = g.gram_iters ? (g.last_gram_rec ? 2 : 3) : 5;
-    const double n_rc = g.gram_iters ? 3 : 5;
-    const double n_rr = g.gram_iters ? (g.last_gram_rec ? 13 : 11) : 5;
-    *ns5_flop = n_gram * r * r * cc + n_rc * 2.0 * r * r * cc + n_rr * r * r * r;
-  }
+  if (ns5_flop) *ns5_flop = ns5_schedule(g.r, g.c, c->gram_span, g.ns_fp32 != 0).flop;
   return PRM_OK;
 }
 
@@ -475,33 +464,33 @@ extern "C" int prm_refresh_segments(prm_ctx* c, const int* mats, int n, const vo
                                     int64_t segment_elems, const int64_t* offsets, int world, int rank,
                                     void* const* param_shards, void* cuda_stream) {
   if (!c) return PRM_ERR_ARG;
-  if (!c->ws) return fail(c, PRM_ERR_WORKSPACE, "prm_refresh_gathered: no workspace attached");
+  if (!c->ws) return fail(c, PRM_ERR_WORKSPACE, "prm_refresh_segments: no workspace attached");
   if (n < 0 || (n > 0 && (!mats || !offsets || !param_shards || !segments)))
-    return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: NULL argument");
-  if (world < 1 || rank < 0 || rank >= world) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: bad world or rank");
-  if (world > kMaxWorld) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: more than 64 ranks");
-  if (segment_elems < 0) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: negative segment size");
+    return fail(c, PRM_ERR_ARG, "prm_refresh_segments: NULL argument");
+  if (world < 1 || rank < 0 || rank >= world) return fail(c, PRM_ERR_ARG, "prm_refresh_segments: bad world or rank");
+  if (world > kMaxWorld) return fail(c, PRM_ERR_ARG, "prm_refresh_segments: more than 64 ranks");
+  if (segment_elems < 0) return fail(c, PRM_ERR_ARG, "prm_refresh_segments: negative segment size");
   SegmentPtrs segs = {};
   bool vec_ok = true;
   for (int q = 0; q < world && n > 0; ++q) {
-    if (!segments[q]) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: NULL segment pointer");
-    if (((uintptr_t)segments[q] & 1) != 0) return fail(c, PRM_ERR_ALIGN, "prm_refresh_gathered: segment not 2-byte aligned");
+    if (!segments[q]) return fail(c, PRM_ERR_ARG, "prm_refresh_segments: NULL segment pointer");
+    if (((uintptr_t)segments[q] & 1) != 0) return fail(c, PRM_ERR_ALIGN, "prm_refresh_segments: segment not 2-byte aligned");
     vec_ok = vec_ok && ((uintptr_t)segments[q] & 15) == 0;
     segs.seg[q] = segments[q];
   }
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   for (int k = 0; k < n; ++k) {
-    if (mats[k] < 0 || mats[k] >= c->n_mats) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: matrix index out of range");
+    if (mats[k] < 0 || mats[k] >= c->n_mats) return fail(c, PRM_ERR_ARG, "prm_refresh_segments: matrix index out of range");
     const Group& g = c->groups[c->group_of_mat[mats[k]]];
     const int64_t chunk = shard_chunk(g.rows, world);
     if (offsets[k] < 0 || offsets[k] + chunk * g.cols > segment_elems)
-      return fail(c, PRM_ERR_SHAPE, "prm_refresh_gathered: a matrix does not fit its segment");
+      return fail(c, PRM_ERR_SHAPE, "prm_refresh_segments: a matrix does not fit its segment");
     int64_t start, count;
     shard_rows(g.rows, world, rank, &start, &count);
     if (count > 0) {
-      if (!param_shards[k]) return fail(c, PRM_ERR_ARG, "prm_refresh_gathered: NULL parameter shard");
+      if (!param_shards[k]) return fail(c, PRM_ERR_ARG, "prm_refresh_segments: NULL parameter shard");
       if (((uintptr_t)param_shards[k] & (c->io_fp32 ? 3 : 1)) != 0)
-        return fail(c, PRM_ERR_ALIGN, "prm_refresh_gathered: parameter shard not aligned to its element size");
+        return fail(c, PRM_ERR_ALIGN, "prm_refresh_segments: parameter shard not aligned to its element size");
     }
   }
   float* fro = (float*)(c->ws + c->off_fro);

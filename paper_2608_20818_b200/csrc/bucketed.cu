@@ -71,9 +71,9 @@ extern "C" int prm_pipeline_model(const double* a, const double* c, int n_bucket
 // Whole matrices assigned to ranks (no optimizer collective at all: every
 // matrix's update is independent of every other's, Algorithm 1 lines 4-10).
 // Longest-processing-time greedy on the refresh cost: matrices in decreasing
-// order of their executed NS5 flop (ties: lower index first) go to the rank
-// with the least load so far (ties: lower rank).  cost_out[q] receives the
-// load of rank q in flop (may be NULL).
+// order of the NS5 flop the default schedule executes for them (ties: lower
+// index first) go to the rank with the least load so far (ties: lower rank).
+// cost_out[q] receives the load of rank q in flop (may be NULL).
 extern "C" int prm_partition_matrices(const int64_t* shapes, int n_mats, int world, int* owner_of_mat,
                                       double* cost_out) {
   if (!shapes || n_mats < 1 || world < 1 || !owner_of_mat) return PRM_ERR_ARG;
@@ -82,8 +82,7 @@ extern "C" int prm_partition_matrices(const int64_t* shapes, int n_mats, int wor
   for (int i = 0; i < n_mats; ++i) {
     const int64_t m = shapes[2 * i], n = shapes[2 * i + 1];
     if (m < 1 || n < 1) return PRM_ERR_SHAPE;
-    const double r = (double)std::min(m, n), c = (double)std::max(m, n);
-    cost[i] = 15.0 * r * r * c + 5.0 * r * r * r;      // printed recurrence with symmetric products
+    cost[i] = ns5_schedule(std::min(m, n), std::max(m, n), 2, std::min(m, n) < kTinyRows).flop;
     order[i] = i;
   }
   std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return cost[a] > cost[b]; });

@@ -186,6 +186,33 @@ struct Group {
 
 inline int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
 
+// Which of the NS5 evaluation orders a matrix with oriented shape r x c takes under
+// PRM_OPT_NS_GRAM_SPAN = span on the tensor-core path, and the flop it executes:
+// X X^T products cost r^2 c (lower blocks only), r x c products 2 r^2 c, symmetric
+// r x r products r^3.
+struct Ns5Schedule {
+  int gram_iters = 0;      // leading iterations on the Gram matrix (0 or kGramIters)
+  int last_gram_rec = 0;   // the last Gram matrix comes from the one before it
+  double flop = 0.0;
+};
+inline Ns5Schedule ns5_schedule(int64_t r, int64_t c, int span, bool fp32_path) {
+  Ns5Schedule s;
+  const int64_t rp = round_up(r, kPad), cp = round_up(c, kPad);
+  // Gram-space iterations trade 6 r^2 (c - r) flop for six r^3 products: worth it from c = 1.5 r
+  // on; below 1024 rows the time is noise and the bf16 rounding of the small r x r matrices
+  // averages less well, so those stay on the printed recurrence.
+  s.gram_iters = (!fp32_path && span && rp >= 1024 && 2 * cp >= 3 * rp) ? kGramIters : 0;
+  // Beyond c = 2r the Gram matrix of the last iteration is also cheaper from the one before it
+  // (A_4 = P_3 A_3 P_3, two r^3 products) than from X_4 (one r^2 c product).
+  s.last_gram_rec = (s.gram_iters && span >= 2 && cp > 2 * rp) ? 1 : 0;
+  const double rd = (double)r, cd = (double)c;
+  const double n_gram = s.gram_iters ? (s.last_gram_rec ? 2 : 3) : 5;
+  const double n_rc = s.gram_iters ? 3 : 5;
+  const double n_rr = s.gram_iters ? (s.last_gram_rec ? 13 : 11) : 5;
+  s.flop = n_gram * rd * rd * cd + n_rc * 2.0 * rd * rd * cd + n_rr * rd * rd * rd;
+  return s;
+}
+
 // dim-0 sharding as torch.chunk does it: rank q of `world` owns stored rows
 // [start, start + count) with chunk = ceil(rows / world).
 inline int64_t shard_chunk(int64_t rows, int world) { return (rows + world - 1) / world; }

@@ -8,7 +8,7 @@
 //   (all-gather by the caller: every rank then holds all segments, rank-major;
 //    or no copy at all: the segments stay where they were written and are
 //    read through peer-mapped pointers)
-//   ns_gather_prepass_kernel  "reconstruct full momenta": reads the rows of a
+//   ns_gather_prepass_kernel  the full-matrix rebuild (line 5): reads the rows of a
 //                             matrix from the segments they arrived in (or
 //                             straight from the owning GPUs' memory) and
 //                             writes the oriented, zero-padded NS5 input X with
@@ -16,7 +16,7 @@
 //                             index arithmetic, no full matrix is assembled
 //                             outside the NS5 workspace
 //   (NS5 products as on one GPU)
-//   ns_slice_update_kernel    "slice the results back to local shards":
+//   ns_slice_update_kernel    each rank keeps its own rows of the result (also line 5):
 //                             W_shard <- (1 - eta lambda) W_shard - eta s X_5
 //                             on this rank's rows only
 //

@@ -380,6 +380,8 @@ def parse_args(argv=None):
     ap.add_argument("--ns5-schedule", type=int, default=2, choices=[0, 1, 2],
                     help="PRM_OPT_NS_GRAM_SPAN: 0 printed recurrence, 1 first three iterations in Gram space, "
                          "2 (library default) also the last Gram matrix from the one before it")
+    ap.add_argument("--tall-kernel", type=int, default=0, choices=[0, 1, 2],
+                    help="PRM_OPT_TALL_KERNEL: 0/1 two passes over the tall matrices, 2 the single-pass streaming kernel")
     ap.add_argument("--partition", default="replicas", choices=["replicas", "matrices"],
                     help="N > 1: independent replicas (weak scaling), or one shape set whose matrices are dealt "
                          "out to the ranks by prm_partition_matrices (strong scaling, no optimizer collective)")
@@ -515,7 +517,7 @@ def main(argv=None):
     opt = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
                                 io_dtype=wl.io_dtype, check_mode=args.check_mode,
                                 gram_span=0 if args.printed_ns5 else args.ns5_schedule,
-                                ns_workspace_bytes=ns_cap, device=dev)
+                                ns_workspace_bytes=ns_cap, tall_kernel=args.tall_kernel, device=dev)
     gram_iters = {(g["rows"], g["cols"]): g["gram_iters"] for g in opt.groups()}
     exec_flop = {(g["rows"], g["cols"]): g["ns5_flop"] for g in opt.groups()}
     params = [make_param(wl, i, dev) for i in range(n)]
@@ -635,6 +637,32 @@ def main(argv=None):
         opt0.close()
         del opt0
 
+    # --------------------------- the other tall-matrix row step beside it
+    # Four row steps with the tall kernel that the main region did not use (two passes / single
+    # pass), same buffers, so that one line carries both.
+    tall_alt = None
+    if any(sh[0] > sh[1] for sh in wl.shapes) and not args.no_printed and wl.io_dtype == "bf16":
+        alt = 1 if args.tall_kernel == 2 else 2
+        torch.cuda.empty_cache()
+        opt1 = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
+                                     io_dtype=wl.io_dtype, ns_workspace_bytes=1, no_refresh=True, tall_kernel=alt,
+                                     device=dev)
+        barrier()
+        for k in range(6):                       # two warm-up row steps, four timed
+            if k == 2:
+                opt1.profile(True)
+            opt1.step(params, grads, moms, 1)
+        barrier()
+        prof1 = opt1.profile_read()
+        assert opt1.status() == B.PRM_OK
+        (alt_ms,) = max_over_ranks([prof1["row_tall"][0] / 4], dev)
+        tall_alt = {"kernel": "single pass (streaming)" if alt == 2 else "two passes", "tall_ms_per_step": alt_ms,
+                    "launches_per_step": prof1["row_tall"][1] // 4,
+                    "note": "four row steps back to back after the main region (no refresh in between: SM clock "
+                            "higher than inside the K-step period)"}
+        opt1.close()
+        del opt1
+
     if rank != 0:
         if dist:
             td.destroy_process_group()
@@ -675,6 +703,7 @@ def main(argv=None):
                    "parallelism": parallelism, "matrices_rank0": n,
                    "device_memory": mem, "ns_workspace_cap_bytes": ns_cap,
                    "gradient_sets": n_sets,
+                   "tall_row_step": "single pass (streaming)" if args.tall_kernel == 2 else "two passes",
                    "l2": "inputs larger than L2 (working set %.1f GB)" % (el * 8 / 1e9),
                    "first_timed_step_index": t_first + args.warmup},
         "refresh_ms": mean_ref if n_ref else None, "row_step_ms": mean_row if n_row else None,
@@ -695,6 +724,9 @@ def main(argv=None):
                            "wide_ms_per_step": prof["row_wide"][0] / n_row, "tall_ms_per_step": prof["row_tall"][0] / n_row,
                            "tall_GB/s": (el_tall * (3 * io_bytes + 8) / (prof["row_tall"][0] / n_row * 1e-3) / 1e9
                                          if prof["row_tall"][0] > 0 else None)}
+        if tall_alt is not None:
+            tall_alt["tall_GB/s"] = el_tall * (3 * io_bytes + 8) / (tall_alt["tall_ms_per_step"] * 1e-3) / 1e9
+            out["row_step"]["other_tall_kernel"] = tall_alt
     if n_ref and gemm_ms > 0:
         tf_exec = ex * n_ref / (gemm_ms * 1e-3) / 1e12
         out["ns5"] = {"TFLOP/s_exec": tf_exec,

@@ -34,6 +34,13 @@ def bf16_round(x):
     return u.astype(np.uint32).view(np.float32).reshape(x.shape)
 
 
+def bf16_split_round(x):
+    """x kept as the sum of two bf16 numbers (hi = bf16(x), lo = bf16(x - hi)): 16 mantissa bits
+    instead of 8, what a product costs three (symmetric) or two tensor-core passes to consume."""
+    hi = bf16_round(x)
+    return hi + bf16_round(np.asarray(x, dtype=np.float32) - hi)
+
+
 def _f32(x):
     return np.asarray(x, dtype=np.float32)
 
@@ -50,9 +57,11 @@ def ns5_fp64(U, eps_ns=1e-7):
     return X
 
 
-def ns5_bf16_printed(U, eps_ns=1e-7, rnd=bf16_round):
+def ns5_bf16_printed(U, eps_ns=1e-7, rnd=bf16_round, rnd_rr=None):
     """Five printed iterations, bf16 storage (rnd), fp32 accumulation.  With
-    rnd = identity this is plain fp32 arithmetic."""
+    rnd = identity this is plain fp32 arithmetic.  rnd_rr, if given, is the
+    storage of the r x r matrices A and B alone."""
+    rnd_rr = rnd if rnd_rr is None else rnd_rr
     U = _f32(U)
     al = np.float32(1.0 / (np.sqrt(np.sum(U.astype(np.float64) ** 2)) + eps_ns))
     X = rnd(U)
@@ -60,8 +69,8 @@ def ns5_bf16_printed(U, eps_ns=1e-7, rnd=bf16_round):
         A = X @ X.T
         if k == 0:
             A = A * (al * al)
-        A = rnd(A)
-        B = rnd(np.float32(NS_B) * A + np.float32(NS_C) * (A @ A))
+        A = rnd_rr(A)
+        B = rnd_rr(np.float32(NS_B) * A + np.float32(NS_C) * (A @ A))
         Xn = np.float32(NS_A) * X + B @ X
         if k == 0:
             Xn = al * Xn
@@ -69,14 +78,15 @@ def ns5_bf16_printed(U, eps_ns=1e-7, rnd=bf16_round):
     return X
 
 
-def ns5_bf16_gramspace(U, last_gram_from_previous, eps_ns=1e-7, rnd=bf16_round):
+def ns5_bf16_gramspace(U, last_gram_from_previous, eps_ns=1e-7, rnd=bf16_round, rnd_x0=None):
     """Iterations 1-3 on the Gram matrix, 4 and 5 as printed; with
     last_gram_from_previous the Gram matrix of iteration 5 is P_3 A_3 P_3
-    instead of X_4 X_4^T."""
+    instead of X_4 X_4^T.  rnd_x0, if given, is the storage of the input X_0
+    alone (it enters two products: X_0 X_0^T and Q X_0)."""
     a, b, c = np.float32(NS_A), np.float32(NS_B), np.float32(NS_C)
     U = _f32(U)
     al = np.float32(1.0 / (np.sqrt(np.sum(U.astype(np.float64) ** 2)) + eps_ns))
-    X0 = rnd(U)
+    X0 = (rnd if rnd_x0 is None else rnd_x0)(U)
 
     def poly(A):
         return rnd(b * A + c * (A @ A))

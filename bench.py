@@ -47,8 +47,9 @@ GEMM_CLASSES = ("gram", "poly", "update", "update_final", "gramspace")
 # DRAM traffic of the kernels, from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum) of a
 # one-block case of the 9B-class set, scaled to a full launch by the work it processes (traffic
 # grows in proportion to it).
-GEMM_DRAM_BYTES_PER_EXEC_FLOP = 1445.6e6 / (8 * 4096 ** 2 * 12288 + 13 * 4096 ** 3)   # all 18 products of one matrix
-ROW_DRAM_BYTES_PER_ELEMENT = {"wide": 14.0, "tall": 20.0}   # the tall matrices take two passes over g and m
+GEMM_DRAM_BYTES_PER_EXEC_FLOP = 1449.7e6 / (8 * 4096 ** 2 * 12288 + 13 * 4096 ** 3)   # all 18 products of one matrix
+ROW_DRAM_BYTES_PER_ELEMENT = {"wide": 14.0, "tall": 20.0,    # the tall matrices take two passes over g and m,
+                              "tall_stream": 13.6}           # one with the streaming kernel
 
 
 # ----------------------------------------------------------------- accounting
@@ -758,7 +759,8 @@ def main(argv=None):
                                "peak_source": "%s sustained bf16 matmul" % pk["source"]}
     elif n_row:
         gbs = row_bytes / (row_kernel_ms / n_row * 1e-3) / 1e9
-        traffic = (ROW_DRAM_BYTES_PER_ELEMENT["wide"] * (el - el_tall) + ROW_DRAM_BYTES_PER_ELEMENT["tall"] * el_tall)
+        tall_key = "tall_stream" if args.tall_kernel == 2 else "tall"
+        traffic = (ROW_DRAM_BYTES_PER_ELEMENT["wide"] * (el - el_tall) + ROW_DRAM_BYTES_PER_ELEMENT[tall_key] * el_tall)
         out["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                            "frac": gbs / pk["hbm_gbs"], "traffic": traffic,
                            "traffic_unit": "DRAM bytes per row step", "kernel": "rowstep_*",

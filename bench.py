@@ -383,6 +383,8 @@ def parse_args(argv=None):
                          "2 (library default) also the last Gram matrix from the one before it")
     ap.add_argument("--tall-kernel", type=int, default=0, choices=[0, 1, 2],
                     help="PRM_OPT_TALL_KERNEL: 0/1 two passes over the tall matrices, 2 the single-pass streaming kernel")
+    ap.add_argument("--split-input", action="store_true",
+                    help="PRM_OPT_NS_SPLIT_INPUT: the NS5 input as two bf16 planes (accuracy option, + 4 r^2 c flop)")
     ap.add_argument("--partition", default="replicas", choices=["replicas", "matrices"],
                     help="N > 1: independent replicas (weak scaling), or one shape set whose matrices are dealt "
                          "out to the ranks by prm_partition_matrices (strong scaling, no optimizer collective)")
@@ -518,7 +520,8 @@ def main(argv=None):
     opt = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
                                 io_dtype=wl.io_dtype, check_mode=args.check_mode,
                                 gram_span=0 if args.printed_ns5 else args.ns5_schedule,
-                                ns_workspace_bytes=ns_cap, tall_kernel=args.tall_kernel, device=dev)
+                                ns_workspace_bytes=ns_cap, tall_kernel=args.tall_kernel, split_input=args.split_input,
+                                device=dev)
     gram_iters = {(g["rows"], g["cols"]): g["gram_iters"] for g in opt.groups()}
     exec_flop = {(g["rows"], g["cols"]): g["ns5_flop"] for g in opt.groups()}
     params = [make_param(wl, i, dev) for i in range(n)]
@@ -705,6 +708,7 @@ def main(argv=None):
                    "device_memory": mem, "ns_workspace_cap_bytes": ns_cap,
                    "gradient_sets": n_sets,
                    "tall_row_step": "single pass (streaming)" if args.tall_kernel == 2 else "two passes",
+                   "ns5_input": "two bf16 planes (PRM_OPT_NS_SPLIT_INPUT)" if args.split_input else "bf16",
                    "l2": "inputs larger than L2 (working set %.1f GB)" % (el * 8 / 1e9),
                    "first_timed_step_index": t_first + args.warmup},
         "refresh_ms": mean_ref if n_ref else None, "row_step_ms": mean_row if n_row else None,

@@ -98,6 +98,24 @@ extern "C" {
  *      the reduced clock that follows a power-capped refresh.
  * Both give the same result up to the order of the fp32 sums.  Before set_workspace. */
 #define PRM_OPT_TALL_KERNEL 13
+/* Accuracy option of the tensor-core NS5 (the paper fixes no arithmetic format for
+ * Eq. app-ns-recurrence; the default stores every operand in bf16).  For inputs whose
+ * spectrum has a few singular values far above the rest, the bf16 rounding of the
+ * NS5 input X_0 alone, whose noise is then of the order of the small singular values,
+ * puts the result 5-6e-2 (relative Frobenius) from the fp64 recurrence.
+ *   0 (default): X_0 stored as one bf16 matrix.
+ *   1: X_0 stored as two bf16 matrices H = bf16(X_0), L = bf16(X_0 - H).  Matrices
+ *      with more than 768 oriented rows take the Gram-space order of
+ *      PRM_OPT_NS_GRAM_SPAN whatever their aspect ratio; in it X_0 enters two
+ *      products only, X_0 X_0^T (computed as H H^T + H L^T + L H^T) and Q X_0
+ *      (Q H + Q L): 4 r^2 c more flop per matrix (+ 25-35 % on the benchmark's
+ *      shapes), one more r x c matrix of workspace per refreshed matrix.  Smaller
+ *      matrices are refreshed in fp32 on CUDA cores, like those with fewer than 64
+ *      rows (the Gram-space order costs them more accuracy on ordinary inputs than
+ *      the second plane returns).  Brings the inputs described above inside the
+ *      2e-2 of all others.  prm_refresh_segments keeps one plane.
+ * Before set_workspace. */
+#define PRM_OPT_NS_SPLIT_INPUT 14
 
 
 typedef struct prm_ctx prm_ctx;

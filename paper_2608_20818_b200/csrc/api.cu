@@ -26,6 +26,7 @@ struct prm_ctx {
   float gamma_ns = 1.f;   // multiplier on the NS5 branch (ablation: "scalar-controlled" uses gamma)
   int no_refresh = 0;     // ablation: RowNorm at every step
   int gram_span = 2;      // NS5 schedule of the tensor-core path (PRM_OPT_NS_GRAM_SPAN)
+  int split_input = 0;    // NS5 input as two bf16 planes (PRM_OPT_NS_SPLIT_INPUT)
   int tall_kernel = 0;    // row step of tall groups (PRM_OPT_TALL_KERNEL): 0 auto, 1 two passes, 2 streaming where possible
 
   std::vector<Group> groups;
@@ -117,13 +118,15 @@ static void compute_layout(prm_ctx* c) {
       g.tall_nu_off = off;      off = align_up(off + (size_t)g.count * g.cols * 4, 256);
       g.tall_sync_off = off;    off = align_up(off + tall_stream_sync_ints(g.cols, g.count) * sizeof(int), 256);
     }
-    g.ns_fp32 = (c->check_mode || g.r < kTinyRows) ? 1 : 0;
+    g.ns_fp32 = (c->check_mode || g.r < kTinyRows || (c->split_input && split_takes_fp32(g.r))) ? 1 : 0;
     const size_t e = g.ns_fp32 ? 4 : 2;
-    const Ns5Schedule sched = ns5_schedule(g.r, g.c, c->gram_span, g.ns_fp32 != 0);
+    g.split = (c->split_input && !g.ns_fp32) ? 1 : 0;
+    const Ns5Schedule sched = ns5_schedule(g.r, g.c, c->gram_span, g.ns_fp32 != 0, g.split != 0);
     g.gram_iters = sched.gram_iters;
     g.last_gram_rec = sched.last_gram_rec;
-    // X ping-pong, A, B (+ two more r x r matrices for the Gram-space iterations)
-    const size_t per_mat = e * (size_t)(2 * g.rp * g.cp + (g.gram_iters ? 4 : 2) * g.rp * g.rp);
+    // X ping-pong (the first buffer twice as large where X_0 is a pair of planes), A, B (+ two
+    // more r x r matrices for the Gram-space iterations)
+    const size_t per_mat = e * (size_t)((g.split ? 3 : 2) * g.rp * g.cp + (g.gram_iters ? 4 : 2) * g.rp * g.rp);
     int nb = (int)std::min<size_t>((size_t)g.count, std::max<size_t>(1, c->ns_cap / per_mat));
     // equal sub-batches: 42 matrices with room for 18 run as 14+14+14, not 18+18+6
     const int chunks = (g.count + nb - 1) / nb;
@@ -213,6 +216,12 @@ extern "C" int prm_set_option(prm_ctx* c, int key, double v) {
       if (attached) return fail(c, PRM_ERR_STATE, "option must be set before prm_set_workspace");
       if (v != 0 && v != 1 && v != 2) return fail(c, PRM_ERR_ARG, "value must be 0, 1 or 2");
       c->tall_kernel = (int)v; return PRM_OK;
+    case PRM_OPT_NS_SPLIT_INPUT:
+      if (attached) return fail(c, PRM_ERR_STATE, "option must be set before prm_set_workspace");
+      if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
+      c->split_input = (int)v;
+      compute_layout(c);
+      return PRM_OK;
     case PRM_OPT_IO_DTYPE:
     case PRM_OPT_CHECK_MODE:
     case PRM_OPT_NS_GRAM_SPAN:
@@ -286,7 +295,7 @@ extern "C" int prm_group_info(const prm_ctx* c, int group, int64_t* rows, int64_
   if (count) *count = g.count;
   if (ns_batch) *ns_batch = g.ns_batch;
   if (gram_iters) *gram_iters = g.gram_iters;
-  if (ns5_flop) *ns5_flop = ns5_schedule(g.r, g.c, c->gram_span, g.ns_fp32 != 0).flop;
+  if (ns5_flop) *ns5_flop = ns5_schedule(g.r, g.c, c->gram_span, g.ns_fp32 != 0, g.split != 0).flop;
   return PRM_OK;
 }
 
@@ -301,17 +310,22 @@ struct NsFinal {
 
 // The NS5 products of one sub-batch of nb matrices of group g whose oriented
 // input U already sits in the first X buffer of the NS5 region, alpha computed.
-// Returns the index (0 or 1) of the X buffer that holds X_5 when fin is null.
-static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFinal* fin, int* x_out,
-                                cudaStream_t stream) {
+// *x_out receives the X buffer that holds X_5 when fin is null.
+// split: X_0 was written as a pair of bf16 planes per matrix (Group::split, Gram-space order
+// only); the first X buffer is then twice as large and is reused as an ordinary X buffer
+// once X_3 exists.
+static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFinal* fin, const char** x_out,
+                                cudaStream_t stream, bool split = false) {
   const size_t e = g.ns_fp32 ? 4 : 2;
   const int64_t rc = g.rp * g.cp, rr = g.rp * g.rp;
   float* alpha = (float*)(c->ws + c->off_alpha);
   int* status = (int*)(c->ws + c->off_status);
   char* base = c->ws + c->off_ns;
-  char* X[2] = {base, base + e * rc * nb};
+  const int x0_planes = g.split ? 2 : 1;           // the layout always leaves room for the pair
+  if (split && (!g.split || !g.gram_iters || g.ns_fp32)) return cudaErrorInvalidValue;
+  char* X[2] = {base, base + (size_t)x0_planes * e * rc * nb};
   char* R[4];                                      // r x r matrices (lower blocks)
-  for (int k = 0; k < 4; ++k) R[k] = base + 2 * e * rc * nb + (size_t)k * e * rr * nb;
+  for (int k = 0; k < 4; ++k) R[k] = base + (size_t)(x0_planes + 1) * e * rc * nb + (size_t)k * e * rr * nb;
   char* A = R[0];
   char* B = R[1];
   cudaError_t ce;
@@ -347,6 +361,7 @@ static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFina
     GemmProblem pa;
     pa.P = X[0]; pa.Q = X[0]; pa.Mp = g.rp; pa.Np = g.rp; pa.Kp = g.cp;
     pa.bs_P = rc; pa.bs_Q = rc; pa.batch = nb; pa.symmetric = 1;
+    if (split) { pa.split = 1; pa.bs_P = pa.bs_Q = 2 * rc; }
     Epilogue ea;
     ea.dst = R[0]; ea.ld_dst = g.rp; ea.bs_dst = rr; ea.alpha = alpha; ea.alpha_pow = 2;
     ce = gemm(pa, ea, PRM_PROF_GRAM);                                                          // A_0
@@ -367,6 +382,7 @@ static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFina
       pu.bs_P = rr; pu.bs_Q = rc; pu.batch = nb; pu.symmetric = 0;
       Epilogue eu;
       eu.k_acc = 1.f; eu.k_aux = a * a * a; eu.aux = X[0]; eu.ld_aux = g.cp; eu.bs_aux = rc;
+      if (split) { pu.split = 1; pu.bs_Q = 2 * rc; eu.bs_aux = 2 * rc; }
       eu.alpha = alpha; eu.alpha_pow = 1;
       eu.dst = X[1]; eu.ld_dst = g.cp; eu.bs_dst = rc;
       ce = gemm(pu, eu, PRM_PROF_UPDATE);
@@ -433,7 +449,7 @@ static cudaError_t ns5_products(prm_ctx* c, const Group& g, int nb, const NsFina
     if ((ce = gemm(pu, eu, it + 1 < kNsIters ? PRM_PROF_UPDATE : PRM_PROF_UPDATE_FINAL)) != cudaSuccess) break;
     cur ^= 1;
   }
-  if (x_out) *x_out = cur;
+  if (x_out) *x_out = X[cur];
   return ce;
 }
 
@@ -447,12 +463,12 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
     cudaError_t ce;
     {
       ProfScope ps(c, PRM_PROF_PREPASS, stream);
-      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, g.ns_fp32, c->ws + c->off_ns, fro, alpha, stream,
-                             &c->launches);
+      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, g.ns_fp32, g.split, c->ws + c->off_ns, fro, alpha,
+                             stream, &c->launches);
     }
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("pre-pass: ") + cudaGetErrorString(ce));
     NsFinal fin{t, first, s.decay, s.lr_s * c->gamma_ns};
-    ce = ns5_products(c, g, nb, &fin, nullptr, stream);
+    ce = ns5_products(c, g, nb, &fin, nullptr, stream, g.split != 0);
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("NS5 product: ") + cudaGetErrorString(ce));
   }
   return PRM_OK;
@@ -519,12 +535,11 @@ extern "C" int prm_refresh_segments(prm_ctx* c, const int* mats, int n, const vo
                                       c->eps_ns, g.ns_fp32, c->ws + c->off_ns, fro, alpha, stream, &c->launches);
       }
       if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("gathered pre-pass: ") + cudaGetErrorString(ce));
-      int xi = 0;
-      ce = ns5_products(c, g, nb, nullptr, &xi, stream);
+      const char* X5 = nullptr;
+      ce = ns5_products(c, g, nb, nullptr, &X5, stream);
       if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("NS5 product: ") + cudaGetErrorString(ce));
       {
         ProfScope ps(c, PRM_PROF_UPDATE_FINAL, stream);
-        const char* X5 = c->ws + c->off_ns + (size_t)xi * e * (size_t)(g.rp * g.cp) * nb;
         ce = launch_ns_slice_update(X5, g.ns_fp32, g, nb, shards.data() + done, row_start, rows_local, c->io_fp32,
                                     decay, lr_s, stream, &c->launches);
       }

@@ -177,6 +177,7 @@ struct Group {
   int gram_iters = 0;           // leading NS5 iterations run in Gram space (0 or kGramIters)
   int last_gram_rec = 0;        // 1: the last iteration's Gram matrix comes from the previous one's
   int ns_fp32 = 0;              // 1: NS5 of this group runs in fp32 on CUDA cores (check mode, or a tiny matrix)
+  int split = 0;                // 1: the NS5 input of this group is kept as two bf16 planes (PRM_OPT_NS_SPLIT_INPUT)
   size_t tall_scratch_off = 0;  // byte offset of column partials (tall groups)
   size_t tall_nu_off = 0;       // byte offset of column norms (tall groups)
   size_t tall_sync_off = 0;     // streaming row step: abort flag, per-wave counters and flags
@@ -195,13 +196,21 @@ struct Ns5Schedule {
   int last_gram_rec = 0;   // the last Gram matrix comes from the one before it
   double flop = 0.0;
 };
-inline Ns5Schedule ns5_schedule(int64_t r, int64_t c, int span, bool fp32_path) {
+// split_input (tensor-core path only): X_0 is held as two bf16 planes; the matrix then takes the
+// Gram-space order whatever its aspect ratio (X_0 must enter two products only and X_1, X_2 must
+// never be rounded for the second plane to pay), and those two products run over both planes:
+// + 4 r^2 c flop.  Below kGramMinRows padded rows the caller refreshes in fp32 instead
+// (split_takes_fp32): there the Gram-space order costs benign inputs more than the planes gain.
+constexpr int64_t kGramMinRows = 1024;
+inline bool split_takes_fp32(int64_t r) { return round_up(r, kPad) < kGramMinRows; }
+inline Ns5Schedule ns5_schedule(int64_t r, int64_t c, int span, bool fp32_path, bool split_input = false) {
   Ns5Schedule s;
   const int64_t rp = round_up(r, kPad), cp = round_up(c, kPad);
+  const bool split = split_input && !fp32_path && rp >= kGramMinRows;
   // Gram-space iterations trade 6 r^2 (c - r) flop for six r^3 products: worth it from c = 1.5 r
   // on; below 1024 rows the time is noise and the bf16 rounding of the small r x r matrices
   // averages less well, so those stay on the printed recurrence.
-  s.gram_iters = (!fp32_path && span && rp >= 1024 && 2 * cp >= 3 * rp) ? kGramIters : 0;
+  s.gram_iters = (!fp32_path && ((span && rp >= kGramMinRows && 2 * cp >= 3 * rp) || split)) ? kGramIters : 0;
   // Beyond c = 2r the Gram matrix of the last iteration is also cheaper from the one before it
   // (A_4 = P_3 A_3 P_3, two r^3 products) than from X_4 (one r^2 c product).
   s.last_gram_rec = (s.gram_iters && span >= 2 && cp > 2 * rp) ? 1 : 0;
@@ -210,6 +219,7 @@ inline Ns5Schedule ns5_schedule(int64_t r, int64_t c, int span, bool fp32_path) 
   const double n_rc = s.gram_iters ? 3 : 5;
   const double n_rr = s.gram_iters ? (s.last_gram_rec ? 13 : 11) : 5;
   s.flop = n_gram * rd * rd * cd + n_rc * 2.0 * rd * rd * cd + n_rr * rd * rd * rd;
+  if (split) s.flop += 4.0 * rd * rd * cd;     // H L^T + L H^T (lower blocks) and Q L
   return s;
 }
 

@@ -55,6 +55,11 @@ struct GemmProblem {
   // P and Q may be two different symmetric matrices (symmetric != 0 then
   // computes the lower blocks of P*Q, which is symmetric when they commute).
   int sym_ops = 0;
+  // Tensor-core path: the input X_0 is a pair of bf16 planes H, L (X_0 = H + L), L directly
+  // after H for every matrix (batch stride 2 * Mp * Kp resp. 2 * Kp * Np elements).  Two
+  // products take it: P = Q = X_0, symmetric (computes H H^T + H L^T + L H^T), and the
+  // N-major Q = X_0 under a symmetric P with aux = X_0 (computes P (H + L) and adds k_aux (H + L)).
+  int split = 0;
 };
 
 cudaError_t launch_rowstep(const PtrTables& t, const Group& g, const StepScalars& s, int io_fp32,
@@ -79,9 +84,10 @@ cudaError_t launch_rowstep_tall_stream(const PtrTables& t, const Group& g, const
 // Momentum update + direction input written to the NS5 workspace as the
 // oriented matrix X (r_p x c_p, zero padded), with per-CTA partial sums of
 // squares, then alpha per matrix.  x_fp32: workspace element type (1: fp32
-// check mode, 0: bf16).
+// check mode, 0: bf16).  split (bf16 workspace only): X is written as the plane
+// pair H = bf16(U), L = bf16(U - H), L directly after H for every matrix.
 cudaError_t launch_ns_prepass(const PtrTables& t, const Group& g, int first, int batch,
-                              const StepScalars& s, int io_fp32, int x_fp32, void* X,
+                              const StepScalars& s, int io_fp32, int x_fp32, int split, void* X,
                               float* fro_partial, float* alpha, cudaStream_t stream,
                               int64_t* launches);
 

@@ -18,11 +18,29 @@ namespace prm {
 constexpr int kPreTile = 64;
 constexpr int kPreThreads = 256;
 
+// Split input (lo_off != 0, bf16 workspace): X is written as two planes, H = bf16(U) at the
+// usual place and L = bf16(U - H) lo_off elements further, so that H + L carries 16 mantissa
+// bits of U into the two NS5 products that read X_0.
+__device__ __forceinline__ float through_storage(float v, const __nv_bfloat16*) {
+  return __bfloat162float(__float2bfloat16_rn(v));
+}
+__device__ __forceinline__ float through_storage(float v, const float*) { return v; }
+template <typename XT_>
+__device__ __forceinline__ void store8_planes(XT_* p, int64_t lo_off, const float (&u)[8]) {
+  store8(p, u);
+  if (lo_off) {
+    float l[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) l[e] = u[e] - through_storage(u[e], p);
+    store8(p + lo_off, l);
+  }
+}
+
 template <typename IO, typename XT_, bool VEC>
 __global__ void __launch_bounds__(kPreThreads)
 ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
                   XT_* __restrict__ straight, int64_t ld_s, int64_t bs_s,
-                  XT_* __restrict__ transposed, int64_t ld_t, int64_t bs_t,
+                  XT_* __restrict__ transposed, int64_t ld_t, int64_t bs_t, int64_t lo_off,
                   float* __restrict__ fro_partial) {
   __shared__ float tile[kPreTile][kPreTile + 1];
   __shared__ float warp_part[kPreThreads / 32];
@@ -73,7 +91,7 @@ ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
       acc += u[e] * u[e];
       tile[lr][tx * 8 + e] = u[e];
     }
-    if (straight != nullptr) store8(ds + (int64_t)row * ld_s + col, u);   // padded extent: always in range
+    if (straight != nullptr) store8_planes(ds + (int64_t)row * ld_s + col, lo_off, u);   // padded extent: always in range
   }
   acc = warp_sum(acc);
   if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
@@ -91,7 +109,7 @@ ns_prepass_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
     float u[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) u[e] = tile[tx * 8 + e][lc];
-    store8(dt + (int64_t)(c0 + lc) * ld_t + r0 + tx * 8, u);
+    store8_planes(dt + (int64_t)(c0 + lc) * ld_t + r0 + tx * 8, lo_off, u);
   }
 }
 
@@ -106,7 +124,7 @@ constexpr int kWideCols = kPreThreads * 8;
 template <typename IO, typename XT_>
 __global__ void __launch_bounds__(kPreThreads)
 ns_prepass_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s,
-                       XT_* __restrict__ X, int64_t ld_x, int64_t bs_x, int prow,
+                       XT_* __restrict__ X, int64_t ld_x, int64_t bs_x, int prow, int64_t lo_off,
                        float* __restrict__ fro_partial) {
   __shared__ float warp_part[kPreThreads / 32];
   const int b = blockIdx.z;
@@ -143,7 +161,7 @@ ns_prepass_wide_kernel(PtrTables t, int first, int rows, int cols, StepScalars s
 #pragma unroll
       for (int e = 0; e < 8; ++e) u[e] = 0.f;
     }
-    if (col < ld_x && row < prow) store8(x + (int64_t)row * ld_x + col, u);
+    if (col < ld_x && row < prow) store8_planes(x + (int64_t)row * ld_x + col, lo_off, u);
   }
   acc = warp_sum(acc);
   if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
@@ -181,19 +199,20 @@ void launch_ns_alpha(const float* fro_partial, int nparts, float eps_ns, float* 
 
 template <typename IO, typename XT_>
 static cudaError_t prepass_inst(const PtrTables& t, const Group& g, int first, int batch,
-                                const StepScalars& s, XT_* X, float* fro_partial, float* alpha,
+                                const StepScalars& s, XT_* X, int split, float* fro_partial, float* alpha,
                                 cudaStream_t stream) {
   // Stored extent padded: wide -> (rp, cp), tall -> (cp, rp).
   const int64_t prow = g.tall ? g.cp : g.rp, pcol = g.tall ? g.rp : g.cp;
   XT_* straight = g.tall ? nullptr : X;
   XT_* transposed = g.tall ? X : nullptr;
-  const int64_t bs = g.rp * g.cp;
+  const int64_t lo_off = split ? g.rp * g.cp : 0;      // the L plane of a matrix follows its H plane
+  const int64_t bs = (split ? 2 : 1) * g.rp * g.cp;
   const bool vec = (g.cols % 8 == 0);
   if (!g.tall && vec) {
     dim3 gw((unsigned)((pcol + kWideCols - 1) / kWideCols), (unsigned)(prow / kWideRows), (unsigned)batch);
     if (gw.y <= 65535 && gw.z <= 65535) {
       ns_prepass_wide_kernel<IO, XT_><<<gw, kPreThreads, 0, stream>>>(t, first, (int)g.rows, (int)g.cols, s, X, pcol, bs,
-                                                                        (int)prow, fro_partial);
+                                                                        (int)prow, lo_off, fro_partial);
       ns_alpha_kernel<<<batch, kPreThreads, 0, stream>>>(fro_partial, (int)(gw.x * gw.y), s.eps_ns, alpha);
       return cudaGetLastError();
     }
@@ -202,25 +221,26 @@ static cudaError_t prepass_inst(const PtrTables& t, const Group& g, int first, i
   if (grid.y > 65535 || grid.z > 65535) return cudaErrorInvalidValue;
   if (vec)
     ns_prepass_kernel<IO, XT_, true><<<grid, kPreThreads, 0, stream>>>(
-        t, first, (int)g.rows, (int)g.cols, s, straight, pcol, bs, transposed, prow, bs, fro_partial);
+        t, first, (int)g.rows, (int)g.cols, s, straight, pcol, bs, transposed, prow, bs, lo_off, fro_partial);
   else
     ns_prepass_kernel<IO, XT_, false><<<grid, kPreThreads, 0, stream>>>(
-        t, first, (int)g.rows, (int)g.cols, s, straight, pcol, bs, transposed, prow, bs, fro_partial);
+        t, first, (int)g.rows, (int)g.cols, s, straight, pcol, bs, transposed, prow, bs, lo_off, fro_partial);
   ns_alpha_kernel<<<batch, kPreThreads, 0, stream>>>(fro_partial, (int)(grid.x * grid.y), s.eps_ns, alpha);
   return cudaGetLastError();
 }
 
 cudaError_t launch_ns_prepass(const PtrTables& t, const Group& g, int first, int batch,
-                              const StepScalars& s, int io_fp32, int x_fp32, void* X,
+                              const StepScalars& s, int io_fp32, int x_fp32, int split, void* X,
                               float* fro_partial, float* alpha, cudaStream_t stream,
                               int64_t* launches) {
   *launches += 2;
+  if (split && x_fp32) return cudaErrorInvalidValue;
   if (io_fp32) {
-    if (x_fp32) return prepass_inst<float, float>(t, g, first, batch, s, (float*)X, fro_partial, alpha, stream);
-    return prepass_inst<float, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, fro_partial, alpha, stream);
+    if (x_fp32) return prepass_inst<float, float>(t, g, first, batch, s, (float*)X, 0, fro_partial, alpha, stream);
+    return prepass_inst<float, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, split, fro_partial, alpha, stream);
   }
-  if (x_fp32) return prepass_inst<__nv_bfloat16, float>(t, g, first, batch, s, (float*)X, fro_partial, alpha, stream);
-  return prepass_inst<__nv_bfloat16, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, fro_partial, alpha, stream);
+  if (x_fp32) return prepass_inst<__nv_bfloat16, float>(t, g, first, batch, s, (float*)X, 0, fro_partial, alpha, stream);
+  return prepass_inst<__nv_bfloat16, __nv_bfloat16>(t, g, first, batch, s, (__nv_bfloat16*)X, split, fro_partial, alpha, stream);
 }
 
 }  // namespace prm

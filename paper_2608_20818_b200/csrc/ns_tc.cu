@@ -220,15 +220,28 @@ __device__ __forceinline__ TileCoord decode_tile(int t, int tiles_per_mat, int s
 // Q_MN and SYM_OPS are compile-time so that each product keeps a main loop
 // with constant descriptor strides (a run-time choice measurably slowed the
 // products that need none).
-template <int Q_MN, int SYM_OPS, int AUX2>
+//
+// SEGS > 1: the input X_0 is held as a pair of bf16 planes, X_0 = H + L with
+// H = bf16(X_0) and L = bf16(X_0 - H), stored one after the other per matrix.
+// The k loop then runs over SEGS segments of kseg stages each:
+//   SEGS = 3 (X_0 X_0^T):  H H^T + H L^T + L H^T  (L L^T, 2^-16 of the result, is dropped);
+//                          segment s reads P from plane (s == 2) and Q from plane (s == 1),
+//                          the maps counting planes as batch items (z = 2b + plane);
+//   SEGS = 2 (Q X_0):      Q H + Q L: the symmetric operand P repeats, the N-major operand's
+//                          k runs on through the rows of H and then of L (mapQ covers both
+//                          planes of a matrix as one 2 Kp-row array); the auxiliary term reads
+//                          both planes as well (mapAux with z = 2b and 2b + 1, one coefficient).
+template <int Q_MN, int SYM_OPS, int AUX2, int SEGS>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__ CUtensorMap mapQ,
                const __grid_constant__ CUtensorMap mapAux, const __grid_constant__ CUtensorMap mapAux2,
                const __grid_constant__ CUtensorMap mapDst,
                const __grid_constant__ CUtensorMap mapSymP, const __grid_constant__ CUtensorMap mapSymQ,
-               int ktiles, int tiles_per_mat, int total_tiles, int symmetric, int mt, Epilogue ep,
+               int ktiles, int kseg, int tiles_per_mat, int total_tiles, int symmetric, int mt, Epilogue ep,
                int* status) {
   constexpr int q_mn = Q_MN, sym_ops = SYM_OPS;
+  static_assert(SEGS == 1 || (SEGS == 3 && !Q_MN && !SYM_OPS && !AUX2) || (SEGS == 2 && Q_MN && SYM_OPS == 1 && AUX2),
+                "split-input products: X_0 X_0^T and Q X_0 only");
   // AUX2: a second auxiliary operand (Epilogue::aux2) travels in the half of
   // the slab buffer that the parameter tile of the final update uses; only the
   // Gram-space products of two symmetric matrices need it.
@@ -289,6 +302,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
       const uint32_t lead_full0 = map_to_rank(&full[0], 0);
       for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
         const TileCoord c = decode_tile(t, tiles_per_mat, symmetric, mt);
+        int seg = 0, ktl = 0;                   // SEGS > 1: segment and stage inside it
         for (int kt = 0; kt < ktiles; ++kt, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1;
@@ -298,22 +312,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           if (rank == 0) mbar_expect_tx(&full[s], 2 * kStageBytes);
           const uint32_t lead_full = lead_full0 + 8u * s;
           const int n0 = c.tj * kBN + (int)rank * (kBN / 2);      // this CTA's 128 rows (columns) of Q
-          const int k0 = kt * kKSub * kBK;
+          const int k0 = (SEGS > 1 ? ktl : kt) * kKSub * kBK;     // k inside the segment
           const int kb = k0 / kPad;                               // the stage's 128 k lie inside one 256-block
           uint8_t* sp = sa;
           uint8_t* sq = sa + kKSub * kBytesA;
-          if ((sym_ops & 1) && kb > (c.ti >> 1)) {
-            tma_load_t_stage(sp, &mapSymP, lead_full, c.ti * kBM, k0, c.b);
+          if (SEGS == 3) {
+            tma_load_k_stage(sp, &mapP, lead_full, k0, c.ti * kBM, 2 * c.b + (seg == 2));
+            tma_load_k_stage(sq, &mapQ, lead_full, k0, n0, 2 * c.b + (seg == 1));
           } else {
-            tma_load_k_stage(sp, &mapP, lead_full, k0, c.ti * kBM, c.b);
+            if ((sym_ops & 1) && kb > (c.ti >> 1)) {
+              tma_load_t_stage(sp, &mapSymP, lead_full, c.ti * kBM, k0, c.b);
+            } else {
+              tma_load_k_stage(sp, &mapP, lead_full, k0, c.ti * kBM, c.b);
+            }
+            if ((sym_ops & 2) && kb > c.tj) {
+              tma_load_t_stage(sq, &mapSymQ, lead_full, n0, k0, c.b);
+            } else if (!q_mn) {
+              tma_load_k_stage(sq, &mapQ, lead_full, k0, n0, c.b);
+            } else {
+              // SEGS == 2: the k rows of the second plane follow those of the first
+              tma_load_t_stage(sq, &mapQ, lead_full, n0, kt * kKSub * kBK, c.b);
+            }
           }
-          if ((sym_ops & 2) && kb > c.tj) {
-            tma_load_t_stage(sq, &mapSymQ, lead_full, n0, k0, c.b);
-          } else if (!q_mn) {
-            tma_load_k_stage(sq, &mapQ, lead_full, k0, n0, c.b);
-          } else {
-            tma_load_t_stage(sq, &mapQ, lead_full, n0, k0, c.b);
-          }
+          if (SEGS > 1 && ++ktl == kseg) { ktl = 0; ++seg; }
         }
       }
       // Drain: every load issued must have landed before shared memory is
@@ -345,6 +366,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
         if (!mbar_wait(&tempty[a], aph ^ 1, abort_flag, status)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t tacc = tmem_base + (uint32_t)a * kBN;
+        int ktl = 0;                            // SEGS > 1: stage inside the segment
         for (int kt = 0; kt < ktiles; ++kt, ++it) {
           const int s = it % kStages;
           const uint32_t ph = (it / kStages) & 1;
@@ -353,7 +375,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           const uint32_t sa = smem0 + (uint32_t)s * kStageBytes;
           // K-major tile: 16 elements = 32 bytes further inside the swizzled row (+2 in 16-byte units);
           // M/N-major tile: 16 k-rows = two 1024-byte atoms further (+128).
-          const int kb = (kt * kKSub * kBK) / kPad;               // the stage's 128 k lie inside one 256-block
+          const int kb = ((SEGS > 1 ? ktl : kt) * kKSub * kBK) / kPad;   // the stage's 128 k lie inside one 256-block
+          if (SEGS > 1 && ++ktl == kseg) ktl = 0;
           const bool a_t = (sym_ops & 1) && kb > (c.ti >> 1);
           const bool b_t = q_mn || ((sym_ops & 2) && kb > c.tj);
           const uint32_t sa_k = a_t ? 128u : 2u, sb_k = b_t ? 128u : 2u;
@@ -392,8 +415,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap mapP, const __grid_constant__
           const int j0 = c.tj * kBN + (int)(g % kSlabs) * kSlabCols;
           uint8_t* buf = ebuf + (size_t)bsel * kEpiBufBytes;
           mbar_expect_tx(&eready[bsel], (has_aux ? kSlabBytes : 0u) + ((fin || AUX2) ? kSlabBytes : 0u));
-          if (has_aux) tma_load_3d(buf, &mapAux, &eready[bsel], j0, c.ti * kBM, c.b);
-          if (AUX2) tma_load_3d(buf + kSlabBytes, &mapAux2, &eready[bsel], j0, c.ti * kBM, c.b);
+          if (SEGS == 2) {               // both planes of X_0 through one map, planes counted as batch items
+            tma_load_3d(buf, &mapAux, &eready[bsel], j0, c.ti * kBM, 2 * c.b);
+            tma_load_3d(buf + kSlabBytes, &mapAux, &eready[bsel], j0, c.ti * kBM, 2 * c.b + 1);
+          } else {
+            if (has_aux) tma_load_3d(buf, &mapAux, &eready[bsel], j0, c.ti * kBM, c.b);
+            if (AUX2) tma_load_3d(buf + kSlabBytes, &mapAux2, &eready[bsel], j0, c.ti * kBM, c.b);
+          }
           if (fin) {
             // Parameter tile into the second slab: as stored (wide), or the
             // transposed region in two 64x64 boxes (tall).  Out-of-range parts read as zero.
@@ -635,15 +663,19 @@ TcContext* tc_create(std::string* err) {
     return nullptr;
   }
   tc->sm_count = prop.multiProcessorCount;
-  ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 0, 0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce == cudaSuccess)
-    ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 3, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 3, 0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce == cudaSuccess)
-    ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 3, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 3, 1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce == cudaSuccess)
-    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 0, 0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce == cudaSuccess)
-    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 1, 0, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (ce == cudaSuccess)
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<0, 0, 0, 3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+  if (ce == cudaSuccess)
+    ce = cudaFuncSetAttribute(gemm_tc_kernel<1, 1, 1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
   if (ce != cudaSuccess) {
     if (err) *err = std::string("cudaFuncSetAttribute: ") + cudaGetErrorString(ce);
     delete tc;
@@ -661,7 +693,7 @@ TcContext* tc_create(std::string* err) {
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   int n_clusters = 0;
-  ce = cudaOccupancyMaxActiveClusters(&n_clusters, gemm_tc_kernel<0, 0, 0>, &cfg);
+  ce = cudaOccupancyMaxActiveClusters(&n_clusters, gemm_tc_kernel<0, 0, 0, 1>, &cfg);
   if (ce != cudaSuccess || n_clusters < 1) {
     if (err) *err = std::string("cudaOccupancyMaxActiveClusters: ") + cudaGetErrorString(ce);
     delete tc;
@@ -787,12 +819,23 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   if (!tc) return cudaErrorInvalidValue;
   if (pb.Mp % kBN != 0 || pb.Np % kBN != 0 || pb.Kp % (kBK * kKSub) != 0) return cudaErrorInvalidValue;
   CUtensorMap mp, mq, maux, maux2, mdst, msp, msq;
-  if (!get_map_kstage(tc, pb.P, pb.Mp, pb.Kp, pb.batch, kBM, &mp)) return cudaErrorInvalidValue;
+  // Split input (GemmProblem::split): the two planes of a matrix follow each other, so a map
+  // over them counts 2 * batch items (K-major operand, auxiliary slabs) or 2 * Kp rows per
+  // item (the N-major operand).
+  const int split = pb.split;
+  if (split) {
+    const bool gram = !pb.q_mn && !pb.sym_ops && pb.symmetric && pb.P == pb.Q && !ep.aux && !ep.aux2 && ep.kind == 0;
+    const bool upd = pb.q_mn && pb.sym_ops == 1 && !pb.symmetric && ep.kind == 0 && ep.aux == pb.Q && !ep.aux2;
+    if (!gram && !upd) return cudaErrorInvalidValue;
+  }
+  const int planes = split ? 2 : 1;
+  if (!get_map_kstage(tc, pb.P, pb.Mp, pb.Kp, (split && !pb.q_mn) ? 2 * pb.batch : pb.batch, kBM, &mp))
+    return cudaErrorInvalidValue;
   if (!pb.q_mn) {
-    if (!get_map_kstage(tc, pb.Q, pb.Np, pb.Kp, pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
+    if (!get_map_kstage(tc, pb.Q, pb.Np, pb.Kp, planes * pb.batch, kBN / 2, &mq)) return cudaErrorInvalidValue;
   } else {
     // Q stored [batch][Kp][Np]: boxes of 64 k-rows x 64 n
-    if (pb.symmetric || !get_map_tstage(tc, pb.Q, pb.Kp, pb.Np, pb.batch, &mq)) return cudaErrorInvalidValue;
+    if (pb.symmetric || !get_map_tstage(tc, pb.Q, planes * pb.Kp, pb.Np, pb.batch, &mq)) return cudaErrorInvalidValue;
   }
   // Epilogue maps (product epilogues only): auxiliary and result slabs of 128
   // rows x 64 columns.
@@ -805,8 +848,8 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
     if (pb.Np != pb.Kp || pb.q_mn || !get_map_tstage(tc, pb.Q, pb.Np, pb.Kp, pb.batch, &msq)) return cudaErrorInvalidValue;
   }
   if (ep.aux && (ep.kind == 0 || ep.param_maps)) {
-    if (ep.bs_aux != pb.Mp * ep.ld_aux) return cudaErrorInvalidValue;
-    if (!get_map(tc, ep.aux, pb.Mp, ep.ld_aux, pb.batch, 128, &maux)) return cudaErrorInvalidValue;
+    if (ep.bs_aux != planes * pb.Mp * ep.ld_aux) return cudaErrorInvalidValue;
+    if (!get_map(tc, ep.aux, pb.Mp, ep.ld_aux, planes * pb.batch, 128, &maux)) return cudaErrorInvalidValue;
   }
   if (ep.aux2) {
     // second auxiliary operand: product epilogues of two symmetric operands only
@@ -843,15 +886,21 @@ cudaError_t launch_gemm_tc(TcContext* tc, const GemmProblem& pb, const Epilogue&
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  const int kt = (int)(pb.Kp / (kBK * kKSub));
-#define PRM_TC_LAUNCH(QMN, SYM, AX2)                                                                              \
-  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<QMN, SYM, AX2>, mp, mq, maux, maux2, mdst, msp, msq, kt,          \
-                            (int)per_mat, (int)total, pb.symmetric, (int)mt, ep, status)
-  if (pb.q_mn && pb.sym_ops == 1) PRM_TC_LAUNCH(1, 1, 0);
-  if (pb.q_mn && !pb.sym_ops) PRM_TC_LAUNCH(1, 0, 0);
-  if (!pb.q_mn && pb.sym_ops == 3 && ep.aux2) PRM_TC_LAUNCH(0, 3, 1);
-  if (!pb.q_mn && pb.sym_ops == 3) PRM_TC_LAUNCH(0, 3, 0);
-  if (!pb.q_mn && !pb.sym_ops) PRM_TC_LAUNCH(0, 0, 0);
+  const int kseg = (int)(pb.Kp / (kBK * kKSub));     // stages per pass over k
+  const int segs = !split ? 1 : (pb.q_mn ? 2 : 3);
+  const int kt = segs * kseg;
+  Epilogue e2 = ep;
+  if (segs == 2) e2.k_aux2 = ep.k_aux;               // both planes of X_0 carry the auxiliary coefficient
+#define PRM_TC_LAUNCH(QMN, SYM, AX2, SG)                                                                          \
+  return cudaLaunchKernelEx(&cfg, gemm_tc_kernel<QMN, SYM, AX2, SG>, mp, mq, maux, maux2, mdst, msp, msq, kt,      \
+                            kseg, (int)per_mat, (int)total, pb.symmetric, (int)mt, e2, status)
+  if (segs == 3) PRM_TC_LAUNCH(0, 0, 0, 3);
+  if (segs == 2) PRM_TC_LAUNCH(1, 1, 1, 2);
+  if (pb.q_mn && pb.sym_ops == 1) PRM_TC_LAUNCH(1, 1, 0, 1);
+  if (pb.q_mn && !pb.sym_ops) PRM_TC_LAUNCH(1, 0, 0, 1);
+  if (!pb.q_mn && pb.sym_ops == 3 && ep.aux2) PRM_TC_LAUNCH(0, 3, 1, 1);
+  if (!pb.q_mn && pb.sym_ops == 3) PRM_TC_LAUNCH(0, 3, 0, 1);
+  if (!pb.q_mn && !pb.sym_ops) PRM_TC_LAUNCH(0, 0, 0, 1);
 #undef PRM_TC_LAUNCH
   return cudaErrorInvalidValue;   // no product of the recurrence needs another combination
 }

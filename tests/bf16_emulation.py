@@ -117,25 +117,33 @@ def rel_fro(got, ref):
     return float(np.linalg.norm(got - ref) / np.linalg.norm(ref))
 
 
-def emulated_error(U, schedule):
+def emulated_error(U, schedule, split_input=False):
     """Relative Frobenius error of the emulated bf16 NS5 of the oriented matrix
     U against the fp64 recurrence.  schedule: "printed", "gram" (iterations 1-3
-    in Gram space) or "gram+rec" (also the last Gram matrix by recurrence)."""
+    in Gram space) or "gram+rec" (also the last Gram matrix by recurrence).
+    split_input: X_0 as the sum of two bf16 numbers (Gram-space orders only)."""
     ref = ns5_fp64(U)
-    if schedule == "printed":
+    if schedule == "fp32":
+        got = ns5_bf16_printed(U, rnd=_f32)
+    elif schedule == "printed":
+        assert not split_input
         got = ns5_bf16_printed(U)
     else:
-        got = ns5_bf16_gramspace(U, schedule == "gram+rec")
+        got = ns5_bf16_gramspace(U, schedule == "gram+rec", rnd_x0=bf16_split_round if split_input else None)
     return rel_fro(got, ref)
 
 
-def library_schedule(shape):
+def library_schedule(shape, split_input=False):
     """The order of evaluation the library's default options pick for a stored
     shape (documented in include/prm.h under PRM_OPT_NS_GRAM_SPAN): padded to
     multiples of 256, Gram space from 1024 oriented rows and c >= 1.5 r on, the
-    last Gram matrix by recurrence where also c > 2r."""
+    last Gram matrix by recurrence where also c > 2r.  With PRM_OPT_NS_SPLIT_INPUT
+    every shape from 1024 padded rows on takes the Gram-space order, the smaller
+    ones run in fp32."""
     r, c = min(shape), max(shape)
     rp, cp = -(-r // 256) * 256, -(-c // 256) * 256
-    if rp >= 1024 and 2 * cp >= 3 * rp:
+    if split_input and rp < 1024:
+        return "fp32"
+    if rp >= 1024 and (split_input or 2 * cp >= 3 * rp):
         return "gram+rec" if cp > 2 * rp else "gram"
     return "printed"

@@ -97,6 +97,32 @@ def test_workspace_scales_with_options():
     B.prm_destroy(h)
 
 
+def test_split_input_option_changes_schedule_flop_and_workspace():
+    """PRM_OPT_NS_SPLIT_INPUT: tensor-core groups from 1024 padded rows on take the Gram-space
+    order, pay 4 r^2 c more flop and one more r x c matrix of workspace; smaller ones go to the
+    fp32 path (printed recurrence)."""
+    shapes = [(2048, 6144), (2048, 2048), (512, 1024), (32, 4096)]
+    h = B.prm_create(shapes, 5, 0.95, True, 1e-3, 0.0)
+    base = [B.prm_group_info(h, g) for g in range(4)]
+    ws0 = B.prm_workspace_bytes(h)
+    B.prm_set_option(h, B.PRM_OPT_NS_SPLIT_INPUT, 1)
+    info = [B.prm_group_info(h, g) for g in range(4)]
+    assert [g["gram_iters"] for g in base] == [3, 0, 0, 0]
+    assert [g["gram_iters"] for g in info] == [3, 3, 0, 0]
+    d = 2048.0
+    assert info[0]["ns5_flop"] == base[0]["ns5_flop"] + 4 * d * d * 6144
+    assert info[1]["ns5_flop"] == 9 * d ** 3 + 11 * d ** 3 + 4 * d ** 3       # Gram space, c = r: no shortcut for A_4
+    assert info[2]["ns5_flop"] == base[2]["ns5_flop"] == 15 * 512.0 ** 2 * 1024 + 5 * 512.0 ** 3
+    assert info[3]["ns5_flop"] == base[3]["ns5_flop"]
+    assert B.prm_workspace_bytes(h) > ws0
+    with pytest.raises(B.PrmError) as e:
+        B.prm_set_option(h, B.PRM_OPT_NS_SPLIT_INPUT, 2)
+    assert e.value.code == B.PRM_ERR_ARG
+    B.prm_set_option(h, B.PRM_OPT_CHECK_MODE, 1)
+    assert [B.prm_group_info(h, g)["gram_iters"] for g in range(4)] == [0] * 4
+    B.prm_destroy(h)
+
+
 def test_group_info_and_gram_span_option():
     shapes = [(2048, 6144), (2048, 2048), (8192, 2048), (2048, 6144), (256, 1024), (1024, 1280)]
     h = B.prm_create(shapes, 5, 0.95, True, 1e-3, 0.0)

@@ -94,7 +94,8 @@ def test_what_would_and_would_not_repair_the_spiked_case():
     small singular values.  With X_0 alone as a hi + lo pair - it enters only X_0 X_0^T and Q X_0
     when the first three iterations run in Gram space - the error falls inside the general
     bound; that costs 4 r^2 c more flop per matrix (about +35 % on the DiT shape sets), so the
-    library does not do it."""
+    library does it only on request (PRM_OPT_NS_SPLIT_INPUT).  In the printed order the second
+    plane returns much less: X_1, rounded to bf16, carries the next largest share of the error."""
     shapes = [(512, 1024), (1024, 3072)]
     for shape, g in zip(shapes, U.structured_grads("spiked", shapes)):
         Ut = direction_input_of(g, shape)
@@ -104,6 +105,29 @@ def test_what_would_and_would_not_repair_the_spiked_case():
         x0_split = E.rel_fro(E.ns5_bf16_gramspace(Ut, True, rnd_x0=E.bf16_split_round), ref)
         assert rr_split >= 0.9 * base, (shape, base, rr_split)
         assert x0_split <= 1.2e-2, (shape, x0_split)
+
+
+def test_gram_space_order_costs_small_matrices_accuracy():
+    """Why PRM_OPT_NS_SPLIT_INPUT, which needs the Gram-space order, sends matrices below 1024
+    padded rows to fp32 instead: on plain Gaussian inputs the Gram-space order (with or without
+    the second plane of X_0) lands at or past 2e-2 there, where the printed order stays inside;
+    from 1024 rows on both orders are at 1e-2."""
+    def worst(r, c, schedule, split, seeds=3):
+        out = 0.0
+        for seed in range(seeds):
+            rng = np.random.default_rng(seed)
+            Ut = E.bf16_round((rng.standard_normal((r, c)) * 1e-3).astype(np.float32))
+            out = max(out, E.emulated_error(Ut, schedule, split))
+        return out
+
+    assert worst(64, 2048, "printed", False) <= 1.5e-2
+    assert worst(64, 2048, "gram", True) >= 2.2e-2
+    assert worst(512, 8192, "gram+rec", True, seeds=2) >= 1.9e-2
+    assert worst(1024, 1024, "gram", True, seeds=2) <= 1.1e-2
+    assert E.library_schedule((512, 8192), split_input=True) == "fp32"
+    assert E.library_schedule((1024, 1024), split_input=True) == "gram"
+    assert E.library_schedule((1024, 1024)) == "printed"
+    assert E.library_schedule((1000, 4096), split_input=True) == "gram+rec"
 
 
 def test_few_rows_scatter_past_the_bound():

@@ -113,7 +113,8 @@ extern "C" {
  *      matrices are refreshed in fp32 on CUDA cores, like those with fewer than 64
  *      rows (the Gram-space order costs them more accuracy on ordinary inputs than
  *      the second plane returns).  Brings the inputs described above inside the
- *      2e-2 of all others.  prm_refresh_segments keeps one plane.
+ *      2e-2 of all others.  prm_refresh_segments keeps one plane: its input is
+ *      the bf16 payload of the exchange, which has no second plane to offer.
  * Before set_workspace. */
 #define PRM_OPT_NS_SPLIT_INPUT 14
 

@@ -237,12 +237,13 @@ def test_bucketed_refresh_needs_a_process_group_for_world_above_one():
 
 
 # ------------------------------------------------------------------- on a GPU
-def _emulate_world(shapes, W, G, M, world, cfg, io, check_mode, bucket_bytes, in_place=False):
+def _emulate_world(shapes, W, G, M, world, cfg, io, check_mode, bucket_bytes, in_place=False, split_input=False):
     """All ranks of `world` one after the other on one device.  Returns full
     (W_new, M_new) as fp64 numpy, shards concatenated."""
     dev = "cuda"
     opt = B.PeriodicRowwiseMuon(shapes, cfg.K, cfg.beta, cfg.nesterov, cfg.lr, cfg.wd, gamma=cfg.gamma,
-                                eps_ns=cfg.eps_ns, scale_mode=cfg.scale_mode, io_dtype=io, check_mode=check_mode)
+                                eps_ns=cfg.eps_ns, scale_mode=cfg.scale_mode, io_dtype=io, check_mode=check_mode,
+                                split_input=split_input)
     bucket_of_mat, offsets, segments = B.prm_bucket_plan(shapes, world, bucket_bytes)
     n = len(shapes)
     cut = lambda x, q, rows: x[slice(*(lambda lo_n: (lo_n[0], lo_n[0] + lo_n[1]))(B.prm_shard_rows(rows, world, q)))]
@@ -329,6 +330,30 @@ def test_sharded_refresh_tensor_cores_against_oracle_and_across_world_sizes(io):
             # after the bf16 rounding of U, ~1e-5 relative); the bf16 roundings of the recurrence then
             # fall differently, which moves the result by a good part of its own rounding noise.
             assert U.rel_fro(Wn[i], Wu[i]) <= 2e-2, (s, U.rel_fro(Wn[i], Wu[i]))
+
+
+@pytest.mark.gpu
+def test_sharded_refresh_on_a_handle_with_split_input():
+    """PRM_OPT_NS_SPLIT_INPUT changes the workspace layout (a second plane of X_0), the order of
+    evaluation (Gram space for every matrix from 1024 padded rows on) and sends smaller matrices
+    to fp32.  The sharded refresh, whose bf16 payload has no second plane, runs on the same handle:
+    one plane, the same layout and schedule."""
+    shapes = GPU_SHAPES + [(1024, 2048), (2048, 1024), (1100, 1100)]
+    cfg = U.oracle_cfg(K=1, beta=0.95, nesterov=True, lr=1.0, wd=0.0, scale_mode=1)
+    W, G, M = U.make_inputs(shapes, 41, "bf16", grad_std=1e-3, mom_std=1e-3)
+    for w in W:
+        w.zero_()
+    first = None
+    for world, cap in ((1, 3 << 20), (3, 1 << 20)):
+        Wn, Mn = _emulate_world(shapes, W, G, M, world, cfg, "bf16", False, bucket_bytes=cap, split_input=True)
+        first = first or Wn
+        for i, s in enumerate(shapes):
+            Wr, Mr = O.step_matrix(U.to_np64(W[i]), U.to_np64(G[i]), U.to_np64(M[i]), 0, cfg)
+            U.assert_elementwise(Mn[i], Mr, False, f"momentum {s}")
+            # below 1024 padded rows: fp32 recurrence on the bf16 payload (its rounding, 2^-9 per
+            # element, is what is left); above: the tensor-core path as without the option
+            assert U.rel_fro(Wn[i], Wr) <= (6e-3 if min(s) <= 768 else 2e-2), (s, world, U.rel_fro(Wn[i], Wr))
+            assert np.array_equal(Wn[i], first[i]), (s, world)
 
 
 @pytest.mark.gpu

@@ -53,3 +53,27 @@ def test_refresh_random_shapes(seed, check_mode):
         U.assert_elementwise(Mg[i], Mr, False, f"momentum {sh}")
         err = U.rel_fro(Wg[i], Wr)
         assert err <= (4e-3 if check_mode else 2e-2), (sh, err)     # bf16 store: 2^-9
+
+
+@pytest.mark.parametrize("seed", [6, 7])
+def test_refresh_split_input_random_large_shapes(seed):
+    """Seeded ragged shapes on both sides of 1024 padded rows, wide and tall, column counts that
+    are and are not multiples of 8, with the two-plane NS5 input: every one within 2e-2."""
+    rng = np.random.default_rng(seed)
+    shapes = []
+    for _ in range(5):
+        r = int(rng.integers(700, 1500))
+        c = int(rng.integers(r, 2600))
+        if rng.integers(0, 2):
+            c = 8 * (c // 8)
+        shapes.append((r, c) if rng.integers(0, 2) else (c, r))
+    cfg = U.oracle_cfg(K=1, nesterov=bool(seed & 1), lr=1.0, wd=0.0)
+    W, G, M = U.make_inputs(shapes, 90 + seed, "bf16", grad_std=1e-3, mom_std=1e-3)
+    for w in W:
+        w.zero_()
+    Wg, Mg = U.gpu_step(shapes, W, G, M, 0, cfg, "bf16", False, split_input=True)
+    for i, sh in enumerate(shapes):
+        Wr, Mr = O.step_matrix(U.to_np64(W[i]), U.to_np64(G[i]), U.to_np64(M[i]), 0, cfg)
+        U.assert_elementwise(Mg[i], Mr, False, f"momentum {sh}")
+        err = U.rel_fro(Wg[i], Wr)
+        assert err <= 2e-2, (sh, err)

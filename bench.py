@@ -383,6 +383,9 @@ def parse_args(argv=None):
                          "2 (library default) also the last Gram matrix from the one before it")
     ap.add_argument("--tall-kernel", type=int, default=0, choices=[0, 1, 2],
                     help="PRM_OPT_TALL_KERNEL: 0/1 two passes over the tall matrices, 2 the single-pass streaming kernel")
+    ap.add_argument("--ns-workspace-gib", type=float, default=None,
+                    help="PRM_OPT_NS_WORKSPACE_BYTES in GiB (library default 8): matrices of a shape are refreshed in "
+                         "sub-batches that fit")
     ap.add_argument("--split-input", action="store_true",
                     help="PRM_OPT_NS_SPLIT_INPUT: the NS5 input as two bf16 planes (accuracy option, + 4 r^2 c flop)")
     ap.add_argument("--partition", default="replicas", choices=["replicas", "matrices"],
@@ -517,6 +520,8 @@ def main(argv=None):
     resident = elements(wl.shapes) * (2 * io_bytes + 4)
     nearly_full = mem is not None and resident > 0.8 * mem["free_gib"] * 2 ** 30
     ns_cap = NS_WORKSPACE_BYTES_WHEN_FULL if nearly_full else None
+    if args.ns_workspace_gib is not None:
+        ns_cap = int(args.ns_workspace_gib * 2 ** 30)
     opt = B.PeriodicRowwiseMuon(wl.shapes, K, wl.beta, wl.nesterov, wl.lr, wl.wd, gamma=wl.gamma,
                                 io_dtype=wl.io_dtype, check_mode=args.check_mode,
                                 gram_span=0 if args.printed_ns5 else args.ns5_schedule,

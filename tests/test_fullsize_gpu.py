@@ -190,3 +190,24 @@ def test_check_mode_direction_at_4096():
         Wr, _ = O.step_matrix(U.to_np64(W[0]), U.to_np64(G[0]), U.to_np64(M[0]), 0, cfg)
         err = U.rel_fro(Wg[0], Wr)
         assert err <= tol, (mode, err)
+
+
+def test_split_input_on_one_block_of_the_9b_class_set():
+    """PRM_OPT_NS_SPLIT_INPUT at the benchmark's matrix sizes: one matrix of every d = 4096 shape,
+    the two-plane tensor-core refresh against the fp32 check mode, and against the fp64 oracle on
+    the square matrix (the one shape whose order of evaluation the option changes)."""
+    d = 4096
+    shapes = [(d, 3 * d), (d, d), (d, 4 * d), (4 * d, d), (d, 6 * d)]
+    cfg = U.oracle_cfg(K=1, beta=0.95, nesterov=True, lr=1.0, wd=0.0, scale_mode=0)
+    W, G, M = U.make_inputs(shapes, 4097, "bf16", grad_std=1e-3, mom_std=1e-3)
+    for w in W:
+        w.zero_()
+    Ws, Ms = U.gpu_step(shapes, W, G, M, 0, cfg, "bf16", False, split_input=True)
+    Wc, Mc = U.gpu_step(shapes, W, G, M, 0, cfg, "bf16", True)
+    for i, s in enumerate(shapes):
+        assert np.array_equal(Ms[i], Mc[i]), s
+        err = U.rel_fro(Ws[i], Wc[i])
+        assert err <= 2e-2, (s, err)
+    Wr, _ = O.step_matrix(U.to_np64(W[1]), U.to_np64(G[1]), U.to_np64(M[1]), 0, cfg)
+    err = U.rel_fro(Ws[1], Wr)
+    assert err <= 2e-2, err

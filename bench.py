@@ -383,6 +383,8 @@ def parse_args(argv=None):
                          "2 (library default) also the last Gram matrix from the one before it")
     ap.add_argument("--tall-kernel", type=int, default=0, choices=[0, 1, 2],
                     help="PRM_OPT_TALL_KERNEL: 0/1 two passes over the tall matrices, 2 the single-pass streaming kernel")
+    ap.add_argument("--wide-kernel", type=int, default=0, choices=[0, 1],
+                    help="PRM_OPT_WIDE_KERNEL: 0 the persistent bulk-copy-fed row step of wide matrices, 1 one row per CTA")
     ap.add_argument("--ns-workspace-gib", type=float, default=None,
                     help="PRM_OPT_NS_WORKSPACE_BYTES in GiB (library default 8): matrices of a shape are refreshed in "
                          "sub-batches that fit")
@@ -526,7 +528,7 @@ def main(argv=None):
                                 io_dtype=wl.io_dtype, check_mode=args.check_mode,
                                 gram_span=0 if args.printed_ns5 else args.ns5_schedule,
                                 ns_workspace_bytes=ns_cap, tall_kernel=args.tall_kernel, split_input=args.split_input,
-                                device=dev)
+                                wide_kernel=args.wide_kernel, device=dev)
     gram_iters = {(g["rows"], g["cols"]): g["gram_iters"] for g in opt.groups()}
     exec_flop = {(g["rows"], g["cols"]): g["ns5_flop"] for g in opt.groups()}
     params = [make_param(wl, i, dev) for i in range(n)]
@@ -713,6 +715,7 @@ def main(argv=None):
                    "device_memory": mem, "ns_workspace_cap_bytes": ns_cap,
                    "gradient_sets": n_sets,
                    "tall_row_step": "single pass (streaming)" if args.tall_kernel == 2 else "two passes",
+                   "wide_row_step": "one row per CTA" if args.wide_kernel == 1 else "persistent, bulk copies",
                    "ns5_input": "two bf16 planes (PRM_OPT_NS_SPLIT_INPUT)" if args.split_input else "bf16",
                    "l2": "inputs larger than L2 (working set %.1f GB)" % (el * 8 / 1e9),
                    "first_timed_step_index": t_first + args.warmup},

@@ -40,6 +40,7 @@ PRM_OPT_NO_REFRESH = 11
 PRM_OPT_NS_GRAM_SPAN = 12
 PRM_OPT_TALL_KERNEL = 13
 PRM_OPT_NS_SPLIT_INPUT = 14
+PRM_OPT_WIDE_KERNEL = 15
 
 EXPORTS = (
     "prm_create", "prm_set_option", "prm_workspace_bytes", "prm_set_workspace", "prm_step",
@@ -388,7 +389,7 @@ class PeriodicRowwiseMuon:
     def __init__(self, shapes, K, beta=0.95, nesterov=False, lr=5e-3, wd=0.01, *, gamma=0.15,
                  eps_row=1e-8, eps_ns=1e-7, scale_mode=1, io_dtype="bf16", check_mode=False,
                  ns_workspace_bytes=None, gamma_ns=1.0, no_refresh=False, gram_span=2, tall_kernel=0,
-                 split_input=False, device="cuda"):
+                 split_input=False, wide_kernel=0, device="cuda"):
         self.shapes = [(int(m), int(n)) for (m, n) in shapes]
         self.device = torch.device(device)
         self.io_dtype = io_dtype
@@ -406,6 +407,7 @@ class PeriodicRowwiseMuon:
             prm_set_option(self.h, PRM_OPT_NS_GRAM_SPAN, int(gram_span))
             prm_set_option(self.h, PRM_OPT_TALL_KERNEL, int(tall_kernel))
             prm_set_option(self.h, PRM_OPT_NS_SPLIT_INPUT, 1 if split_input else 0)
+            prm_set_option(self.h, PRM_OPT_WIDE_KERNEL, int(wide_kernel))
             if ns_workspace_bytes is not None:
                 prm_set_option(self.h, PRM_OPT_NS_WORKSPACE_BYTES, ns_workspace_bytes)
             nbytes = prm_workspace_bytes(self.h)

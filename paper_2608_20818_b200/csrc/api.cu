@@ -27,6 +27,7 @@ struct prm_ctx {
   int no_refresh = 0;     // ablation: RowNorm at every step
   int gram_span = 2;      // NS5 schedule of the tensor-core path (PRM_OPT_NS_GRAM_SPAN)
   int split_input = 0;    // NS5 input as two bf16 planes (PRM_OPT_NS_SPLIT_INPUT)
+  int wide_kernel = 0;    // row step of wide groups (PRM_OPT_WIDE_KERNEL): 0 persistent kernel where it applies, 1 one row per CTA
   int tall_kernel = 0;    // row step of tall groups (PRM_OPT_TALL_KERNEL): 0 auto, 1 two passes, 2 streaming where possible
 
   std::vector<Group> groups;
@@ -212,6 +213,9 @@ extern "C" int prm_set_option(prm_ctx* c, int key, double v) {
     case PRM_OPT_NO_REFRESH:
       if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
       c->no_refresh = (int)v; return PRM_OK;
+    case PRM_OPT_WIDE_KERNEL:
+      if (v != 0 && v != 1) return fail(c, PRM_ERR_ARG, "value must be 0 or 1");
+      c->wide_kernel = (int)v; return PRM_OK;
     case PRM_OPT_TALL_KERNEL:
       if (attached) return fail(c, PRM_ERR_STATE, "option must be set before prm_set_workspace");
       if (v != 0 && v != 1 && v != 2) return fail(c, PRM_ERR_ARG, "value must be 0, 1 or 2");
@@ -671,6 +675,9 @@ static int step_impl(prm_ctx* c, void* const* params, void* const* grads_dev,
                                         (float*)(c->ws + g.tall_scratch_off), (float*)(c->ws + g.tall_nu_off),
                                         (int*)(c->ws + g.tall_sync_off), (int*)(c->ws + c->off_status),
                                         tc_sm_count(c->tc), stream, &c->launches);
+      else if (!g.tall && c->wide_kernel != 1 && tc_sm_count(c->tc) > 0 && wide_stream_takes(g, c->io_fp32))
+        ce = launch_rowstep_wide_stream(t, g, s, tc_sm_count(c->tc), (int*)(c->ws + c->off_status), stream,
+                                        &c->launches);
       else
         ce = launch_rowstep(t, g, s, c->io_fp32, (float*)(c->ws + g.tall_scratch_off),
                             (float*)(c->ws + g.tall_nu_off), stream, &c->launches);

@@ -66,6 +66,12 @@ cudaError_t launch_rowstep(const PtrTables& t, const Group& g, const StepScalars
                            float* tall_partial, float* tall_nu, cudaStream_t stream,
                            int64_t* launches);
 
+// Persistent, bulk-copy-fed row step of a wide group (rowstep_wide_stream.cu): bf16 parameters and
+// gradients, cols % 8 == 0, at most 24576 columns; n_cta CTAs, one per SM.
+bool wide_stream_takes(const Group& g, int io_fp32);
+cudaError_t launch_rowstep_wide_stream(const PtrTables& t, const Group& g, const StepScalars& s, int n_cta, int* status,
+                                       cudaStream_t stream, int64_t* launches);
+
 // Streaming row step of a tall group (rowstep_stream.cu): one pass over HBM,
 // bf16 parameters and gradients with cols % 8 == 0.  maps_dev: three 128-byte
 // tensor maps per matrix of the group (gradient, momentum, parameters; boxes of

@@ -97,6 +97,16 @@ def test_workspace_scales_with_options():
     B.prm_destroy(h)
 
 
+def test_wide_kernel_option_values():
+    h = B.prm_create([(8, 16)], 2, 0.95, False, 1e-3, 0.0)
+    B.prm_set_option(h, B.PRM_OPT_WIDE_KERNEL, 1)
+    B.prm_set_option(h, B.PRM_OPT_WIDE_KERNEL, 0)
+    with pytest.raises(B.PrmError) as e:
+        B.prm_set_option(h, B.PRM_OPT_WIDE_KERNEL, 2)
+    assert e.value.code == B.PRM_ERR_ARG
+    B.prm_destroy(h)
+
+
 def test_split_input_option_changes_schedule_flop_and_workspace():
     """PRM_OPT_NS_SPLIT_INPUT: tensor-core groups from 1024 padded rows on take the Gram-space
     order, pay 4 r^2 c more flop and one more r x c matrix of workspace; smaller ones go to the

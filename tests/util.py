@@ -75,14 +75,14 @@ def oracle_cfg(**kw):
 
 
 def gpu_step(shapes, W, G, M, t, cfg, io, check_mode, ns_workspace_bytes=None, steps=1, grads_fn=None,
-             gram_span=2, tall_kernel=0, launches=None, split_input=False):
+             gram_span=2, tall_kernel=0, launches=None, split_input=False, wide_kernel=0):
     """Run `steps` steps from step index t on the GPU through the C ABI.
     Returns (W_new list, M_new list) as fp64 numpy, after checking canaries."""
     opt = B.PeriodicRowwiseMuon(shapes, cfg.K, cfg.beta, cfg.nesterov, cfg.lr, cfg.wd, gamma=cfg.gamma,
                                 eps_row=cfg.eps_row, eps_ns=cfg.eps_ns, scale_mode=cfg.scale_mode,
                                 io_dtype=io, check_mode=check_mode, ns_workspace_bytes=ns_workspace_bytes,
                                 gamma_ns=cfg.gamma_ns, no_refresh=cfg.no_refresh, gram_span=gram_span,
-                                tall_kernel=tall_kernel, split_input=split_input)
+                                tall_kernel=tall_kernel, split_input=split_input, wide_kernel=wide_kernel)
     gw = [Guarded(w) for w in W]
     gg = [Guarded(g) for g in G]
     gm = [Guarded(m) for m in M]

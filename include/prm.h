@@ -117,13 +117,15 @@ extern "C" {
  *      the bf16 payload of the exchange, which has no second plane to offer.
  * Before set_workspace. */
 #define PRM_OPT_NS_SPLIT_INPUT 14
-/* Which kernel takes the row step (rho_t = 0) of WIDE matrices (Eq. rownorm on stored rows):
- *   0 (default): for bf16 matrices with cols % 8 == 0 and at most 24576 columns a persistent
- *      kernel, one CTA per SM, whose producer warp streams the rows in with bulk asynchronous
- *      copies ahead of the warps that reduce and update them; the kernels of 1 for the rest.
- *   1: one stored row per CTA (per cluster beyond 32768 columns), loads held in registers.
- * Same arithmetic, 14 bytes per element either way; the sums of a row are added in another
- * order, so the two agree to rounding, not bit for bit.  May be changed between steps. */
+/* Which kernels take the row step (rho_t = 0) of WIDE matrices (Eq. rownorm on stored rows)
+ * and their NS5 pre-pass (momentum update, direction input, Frobenius sum):
+ *   0 (default): for bf16 matrices with cols % 8 == 0 (row step: at most 24576 columns)
+ *      persistent kernels, one CTA per SM, whose producer warp streams the rows in with bulk
+ *      asynchronous copies ahead of the warps that work on them; the kernels of 1 for the rest.
+ *   1: row step with one stored row per CTA (per cluster beyond 32768 columns), pre-pass with
+ *      4 rows x 2048 columns per CTA; loads held in registers.
+ * Same arithmetic and bytes per element either way; sums are added in another order, so the
+ * two agree to rounding, not bit for bit.  May be changed between steps. */
 #define PRM_OPT_WIDE_KERNEL 15
 
 

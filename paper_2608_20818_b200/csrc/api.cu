@@ -135,9 +135,10 @@ static void compute_layout(prm_ctx* c) {
     g.ns_batch = nb;
 
     ns_max = std::max(ns_max, per_mat * nb);
-    // one partial per CTA of the pre-pass: 64 x 64 tiles (tall), or 4 rows x 2048 columns (wide)
-    fro_max = std::max(fro_max, (size_t)nb * std::max((size_t)((g.rp / 64) * (g.cp / 64)),
-                                                      (size_t)((g.rp / 4) * ((g.cp + 2047) / 2048))));
+    // one partial per CTA of the pre-pass: 64 x 64 tiles (tall), 4 rows x 2048 columns (wide), or
+    // one per CTA of the persistent kernel (at most 256)
+    fro_max = std::max(fro_max, (size_t)nb * std::max({(size_t)((g.rp / 64) * (g.cp / 64)),
+                                                       (size_t)((g.rp / 4) * ((g.cp + 2047) / 2048)), (size_t)256}));
     batch_max = std::max(batch_max, nb);
   }
   c->off_fro = off;   off = align_up(off + fro_max * 4, 256);
@@ -467,8 +468,19 @@ static int refresh_group(prm_ctx* c, const Group& g, const PtrTables& t, StepSca
     cudaError_t ce;
     {
       ProfScope ps(c, PRM_PROF_PREPASS, stream);
-      ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, g.ns_fp32, g.split, c->ws + c->off_ns, fro, alpha,
-                             stream, &c->launches);
+      const int n_sm = tc_sm_count(c->tc);
+      if (c->wide_kernel != 1 && n_sm > 0 && prepass_stream_takes(g, c->io_fp32, g.ns_fp32)) {
+        ce = launch_ns_prepass_stream(t, g, first, nb, s, g.split, c->ws + c->off_ns, fro, n_sm,
+                                      (int*)(c->ws + c->off_status), stream);
+        if (ce == cudaSuccess) {
+          launch_ns_alpha(fro, prepass_stream_parts(n_sm, g.rp, nb), s.eps_ns, alpha, nb, stream);
+          ce = cudaGetLastError();
+        }
+        c->launches += 2;
+      } else {
+        ce = launch_ns_prepass(t, g, first, nb, s, c->io_fp32, g.ns_fp32, g.split, c->ws + c->off_ns, fro, alpha,
+                               stream, &c->launches);
+      }
     }
     if (ce != cudaSuccess) return fail(c, PRM_ERR_CUDA, std::string("pre-pass: ") + cudaGetErrorString(ce));
     NsFinal fin{t, first, s.decay, s.lr_s * c->gamma_ns};

@@ -97,6 +97,14 @@ cudaError_t launch_ns_prepass(const PtrTables& t, const Group& g, int first, int
                               float* fro_partial, float* alpha, cudaStream_t stream,
                               int64_t* launches);
 
+// The same pre-pass for wide groups with bf16 gradients and workspace and cols % 8 == 0, as a
+// persistent bulk-copy-fed kernel (ns_prepass_stream.cu); n_cta CTAs, one per SM.  Leaves
+// prepass_stream_parts() partials per matrix in fro_partial; the caller runs launch_ns_alpha.
+bool prepass_stream_takes(const Group& g, int io_fp32, int x_fp32);
+int prepass_stream_parts(int n_cta, int64_t prow, int batch);
+cudaError_t launch_ns_prepass_stream(const PtrTables& t, const Group& g, int first, int batch, const StepScalars& s,
+                                     int split, void* X, float* fro_partial, int n_cta, int* status, cudaStream_t stream);
+
 // alpha[b] = 1/(sqrt(sum of nparts partials of matrix b) + eps_ns).
 void launch_ns_alpha(const float* fro_partial, int nparts, float eps_ns, float* alpha, int batch,
                      cudaStream_t stream);

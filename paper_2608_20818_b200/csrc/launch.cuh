@@ -5,6 +5,20 @@
 
 namespace prm {
 
+// cudaFuncSetAttribute holds per device: remembers, per kernel (one object per call site), on
+// which devices the attribute has been set.
+struct PerDeviceOnce {
+  bool done[64] = {};
+  // True if the caller still has to set the attribute on the current device.
+  bool need(int* dev_out) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *dev_out = -1; return true; }
+    *dev_out = dev;
+    return !done[dev];
+  }
+  void mark(int dev) { if (dev >= 0) done[dev] = true; }
+};
+
 // Epilogue of every NS5 product D[i,j] = sum_k P[i,k]*Q[j,k].  With
 // f = alpha[b]^alpha_pow (1 if alpha is null) and
 // v = f*(k_acc*D[i,j] + k_aux*aux[i,j]):

@@ -192,7 +192,7 @@ __global__ void __launch_bounds__(kThreads, 1) ns_prepass_wide_stream_kernel(con
   while (cur < a.batch) { flush(cur); ++cur; }
 }
 
-bool g_ready = false;
+PerDeviceOnce g_ready;
 
 }  // namespace
 
@@ -207,10 +207,11 @@ cudaError_t launch_ns_prepass_stream(const PtrTables& t, const Group& g, int fir
                                      int split, void* X, float* fro_partial, int n_cta, int* status, cudaStream_t stream) {
   if (!prepass_stream_takes(g, 0, 0) || n_cta < 1) return cudaErrorInvalidValue;
   cudaError_t ce;
-  if (!g_ready) {
+  int dev;
+  if (g_ready.need(&dev)) {
     ce = cudaFuncSetAttribute(ns_prepass_wide_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
     if (ce != cudaSuccess) return ce;
-    g_ready = true;
+    g_ready.mark(dev);
   }
   PreArgs a;
   a.t = t; a.first = first; a.batch = batch; a.rows = (int)g.rows; a.cols = (int)g.cols;

@@ -432,7 +432,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) rowstep_tall_stream_kernel(
   if (threadIdx.x == 0 && *abort_flag) atomicExch(abort_g, 1);   // let the other CTAs leave their flag waits at once
 }
 
-bool g_stream_ready = false;
+PerDeviceOnce g_stream_ready;
 
 }  // namespace
 
@@ -465,12 +465,13 @@ cudaError_t launch_rowstep_tall_stream(const PtrTables& t, const Group& g, const
                                        int* sync, int* status, int n_cta, cudaStream_t stream, int64_t* launches) {
   if (!plan.ok) return cudaErrorInvalidValue;
   cudaError_t ce;
-  if (!g_stream_ready) {
+  int dev;
+  if (g_stream_ready.need(&dev)) {
     ce = cudaFuncSetAttribute(rowstep_tall_stream_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
     if (ce == cudaSuccess)
       ce = cudaFuncSetAttribute(rowstep_tall_stream_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
     if (ce != cudaSuccess) return ce;
-    g_stream_ready = true;
+    g_stream_ready.mark(dev);
   }
   ce = cudaMemsetAsync(sync, 0, tall_stream_sync_ints(g.cols, g.count) * sizeof(int), stream);
   if (ce != cudaSuccess) return ce;

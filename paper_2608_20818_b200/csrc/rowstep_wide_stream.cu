@@ -243,15 +243,16 @@ __global__ void __launch_bounds__(kThreads, 1) rowstep_wide_stream_kernel(const 
 
 template <int VPT>
 cudaError_t launch_inst(const WideArgs& a, int n_cta, cudaStream_t stream) {
-  static bool ready[2] = {false, false};
+  static PerDeviceOnce ready[2];
   const int nest = a.s.nesterov ? 1 : 0;
   const size_t smem = wide_smem_bytes<VPT>();
   cudaError_t ce;
-  if (!ready[nest]) {
+  int dev;
+  if (ready[nest].need(&dev)) {
     ce = nest ? cudaFuncSetAttribute(rowstep_wide_stream_kernel<VPT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)
               : cudaFuncSetAttribute(rowstep_wide_stream_kernel<VPT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (ce != cudaSuccess) return ce;
-    ready[nest] = true;
+    ready[nest].mark(dev);
   }
   const int grid = (int)std::min<int64_t>(n_cta, a.total_rows);
   if (nest) rowstep_wide_stream_kernel<VPT, true><<<grid, kThreads, smem, stream>>>(a);

@@ -94,6 +94,22 @@ def test_rowstep_zero_and_tiny_rows():
     np.testing.assert_allclose(Wg[0][0], (1 - 5e-3 * 0.01) * U.to_np64(W[0])[0], rtol=1e-6)
 
 
+@pytest.mark.parametrize("wide_kernel", [0, 1])
+def test_rowstep_zero_and_tiny_rows_bf16(wide_kernel):
+    """The same degenerate rows through the bf16 kernels (persistent and one row per CTA): a zero
+    row only decays, a tiny row is divided by eps_row, a row of one huge element keeps its sign."""
+    shapes = [(6, 4104)]
+    cfg = U.oracle_cfg(K=4, nesterov=True, lr=5e-3, wd=0.01, eps_row=1e-3)
+    W, G, M = U.make_inputs(shapes, 17, "bf16")
+    G[0][0].zero_(); M[0][0].zero_()
+    G[0][1].zero_(); M[0][1].zero_(); G[0][1, 7] = 1e-6
+    G[0][2].zero_(); M[0][2].zero_(); G[0][2, 4100] = -3e4
+    Wg, Mg = U.gpu_step(shapes, W, G, M, 1, cfg, "bf16", True, wide_kernel=wide_kernel)
+    Wr, Mr = O.step_matrix(U.to_np64(W[0]), U.to_np64(G[0]), U.to_np64(M[0]), 1, cfg)
+    U.assert_elementwise(Wg[0], Wr, True, "param")
+    U.assert_elementwise(Mg[0], Mr, False, "momentum")
+
+
 def test_rowstep_run_to_run_bit_identical():
     shapes = [(300, 2056), (1000, 264), (6, 32776)]
     cfg = U.oracle_cfg(K=4, nesterov=True)
